@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the step-attention hot path (RoPE-append -> split-KV attention -> combine).
+
+A "step" is one pass of the whole path for one transformer layer on the 7B-class workload
+(28 query / 4 kv heads, head_dim 128, L = 4096 cached tokens, n = 196 new tokens, bf16).
+The run cycles over a ring of independent layer caches whose footprint exceeds the L2, the
+way a 28-layer model revisits each layer's cache once per navigation step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas (the path has no exchange step); the
+printed value is the max over ranks.  One JSON line goes to stdout on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2512_10310_b200 import workloads as W
+
+RING_LAYERS = 32            # independent layer caches cycled through (footprint > L2)
+L2_BYTES = 126 * 2 ** 20
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+
+class LayerRing:
+    """Device buffers of RING_LAYERS independent layers of the workload + pinned host copies."""
+
+    def __init__(self, B, handle, cfg, dev, layers):
+        self.B, self.h, self.cfg, self.dev = B, handle, cfg, dev
+        L, n, Hq, Hkv, D = cfg.cache_len, cfg.num_new, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
+        self.p = B.step_params(cfg.dtype, Hq, Hkv, D, L, n, L + n, cfg.rope_theta)
+        qbytes = B.evlnStepQRotSize(handle, self.p)
+        wbytes = B.evlnStepWorkspaceSize(handle, self.p)
+        self.splits = B.evlnStepNumSplits(handle, self.p)
+        self.layers = []
+        dt = cfg.torch_dtype
+        for l in range(layers):
+            x = W.make_step_inputs(dataclasses.replace(cfg, seed=cfg.seed * 7919 + l))
+            kc = torch.zeros((Hkv, L + n, D), dtype=dt, device=dev)
+            vc = torch.zeros((Hkv, L + n, D), dtype=dt, device=dev)
+            kc[:, :L] = x["k_cache"].to(dev).permute(1, 0, 2)
+            vc[:, :L] = x["v_cache"].to(dev).permute(1, 0, 2)
+            host_in = [x[s].contiguous().pin_memory() for s in ("q_new", "k_new", "v_new")]
+            self.layers.append(dict(
+                kc=kc, vc=vc, q=x["q_new"].to(dev), k=x["k_new"].to(dev), v=x["v_new"].to(dev),
+                q_rot=torch.empty(qbytes, dtype=torch.uint8, device=dev),
+                ws=torch.empty(wbytes, dtype=torch.uint8, device=dev),
+                out=torch.empty((n, Hq, D), dtype=dt, device=dev),
+                host_in=host_in,
+                host_out=torch.empty((n, Hq, D), dtype=dt).pin_memory(),
+            ))
+        self.bytes_per_layer = 2 * kc.numel() * kc.element_size()
+
+    def step(self, l):
+        B, y = self.B, self.layers[l]
+        B.evlnRopeAppend(self.h, self.p, y["q"], y["k"], y["v"], y["q_rot"], y["kc"], y["vc"])
+        B.evlnStepAttention(self.h, self.p, y["q_rot"], y["kc"], y["vc"], y["ws"])
+        B.evlnStepCombine(self.h, self.p, y["ws"], y["out"], None)
+
+    def attention_only(self, l):
+        y = self.layers[l]
+        self.B.evlnStepAttention(self.h, self.p, y["q_rot"], y["kc"], y["vc"], y["ws"])
+
+    def step_e2e(self, l):
+        """Host buffers in, host buffer out: the copies ride the same stream as the kernels."""
+        y = self.layers[l]
+        for dst, src in zip((y["q"], y["k"], y["v"]), y["host_in"]):
+            dst.copy_(src, non_blocking=True)
+        self.step(l)
+        y["host_out"].copy_(y["out"], non_blocking=True)
+
+
+def capture(fn, layers):
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for l in range(layers):
+            fn(l)                                    # warm the path on the side stream
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g):
+        for l in range(layers):
+            fn(l)
+    return g
+
+
+def timed(run_chunk, chunks, barrier):
+    """Barrier + sync, CUDA events around `chunks` calls of run_chunk on the current stream."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(chunks):
+        run_chunk()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1)            # ms
+
+
+def run_ours(args, rank, world, local_rank, dist):
+    from paper_2512_10310_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    cfg = W.STEP_7B
+    handle = B.evlnCreate(local_rank)
+    ring = LayerRing(B, handle, cfg, dev, RING_LAYERS)
+    for l in range(RING_LAYERS):
+        ring.step(l)
+    assert B.evlnGetDeviceStatus(handle) == 0
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    steps = max(RING_LAYERS, (args.steps // RING_LAYERS) * RING_LAYERS)
+    warm = max(3 * RING_LAYERS, -(-args.warmup // RING_LAYERS) * RING_LAYERS)
+    g_step = capture(ring.step, RING_LAYERS)
+    g_attn = capture(ring.attention_only, RING_LAYERS)
+
+    for _ in range(warm // RING_LAYERS):
+        g_step.replay()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    ms = timed(g_step.replay, steps // RING_LAYERS, barrier)
+    ms_attn = timed(g_attn.replay, steps // RING_LAYERS, barrier)
+    clocks = sampler.stop()
+    assert B.evlnGetDeviceStatus(handle) == 0, "a kernel gave up on a bounded wait"
+
+    # end to end through the public calls with host buffers (eager launches + copies)
+    e2e_steps = min(steps, 64 * RING_LAYERS)
+    for l in range(RING_LAYERS):
+        ring.step_e2e(l)
+    torch.cuda.synchronize()
+
+    def e2e_chunk():
+        for l in range(RING_LAYERS):
+            ring.step_e2e(l)
+    ms_e2e = timed(e2e_chunk, e2e_steps // RING_LAYERS, barrier)
+
+    us_step = max_over_ranks(ms * 1e3 / steps)
+    us_attn = max_over_ranks(ms_attn * 1e3 / steps)
+    us_e2e = max_over_ranks(ms_e2e * 1e3 / e2e_steps)
+    B.evlnDestroy(handle)
+    if rank != 0:
+        return None
+
+    peaks, peaks_kind = load_peaks()
+    flops = cfg.flops()
+    abytes = cfg.algorithmic_bytes()
+    t_flop_us = flops / (peaks["bf16_tflops"] * 1e12) * 1e6
+    t_hbm_us = abytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+    achieved_tf = flops / (us_attn * 1e-6) / 1e12
+    h2d = sum(t.numel() * t.element_size() for t in ring.layers[0]["host_in"])
+    d2h = ring.layers[0]["host_out"].numel() * ring.layers[0]["host_out"].element_size()
+    line = {
+        "metric": "new-frame step-attention latency", "value": round(us_step, 3), "unit": "us/step",
+        "n_gpus": world, "steps": steps, "warmup": warm, "ms_per_step": us_step / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {
+            "workload": f"{cfg.name}: 28q/4kv heads, head_dim 128, L=4096, n=196, theta 1e6, bf16, one layer-step "
+                        "= evlnRopeAppend + evlnStepAttention + evlnStepCombine",
+            "kv_splits": ring.splits,
+            "launch": f"CUDA graph of {RING_LAYERS} layer-steps, replayed",
+            "l2": f"inputs larger than L2: ring of {RING_LAYERS} independent layer caches, "
+                  f"{RING_LAYERS * ring.bytes_per_layer / 2**20:.0f} MiB of K/V revisited round-robin",
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+        },
+        "tflops": round(flops / (us_step * 1e-6) / 1e12 * world, 2),
+        "gbs": round(abytes / (us_step * 1e-6) / 1e9 * world, 1),
+        "steps_per_s": round(world / (us_step * 1e-6), 1),
+        "step_roofline_frac": round(max(t_flop_us, t_hbm_us) / us_step, 4),
+        "roofline": {
+            "kernel": "attn_tc_kernel (evlnStepAttention)", "bound": "tensor",
+            "achieved": round(achieved_tf, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": round(achieved_tf / peaks["bf16_tflops"], 4), "peak_kind": f"{peaks_kind} burst bf16",
+            "traffic": None, "us_per_launch": round(us_attn, 3),
+            "timing": f"CUDA events around graph replays of {RING_LAYERS} back-to-back attention launches",
+            "flops_per_launch": flops,
+        },
+        "e2e": {"value": round(us_e2e, 3), "unit": "us/step", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": 3 * steps,
+        "clocks": clocks,
+    }
+    return line
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arms
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_time(cfg, rows_per_step, steps, warmup):
+    """Times the oracle, as it stands, on `rows_per_step` (token, all-heads-of-one-group) samples."""
+    from oracle import step_oracle as so
+    x = W.make_step_inputs(cfg)
+    f64 = lambda t: np.ascontiguousarray(t.to(torch.float64).numpy())
+    L, n = cfg.cache_len, cfg.num_new
+    kc = np.zeros((L + n, cfg.num_kv_heads, cfg.head_dim))
+    vc = np.zeros_like(kc)
+    kc[:L], vc[:L] = f64(x["k_cache"]), f64(x["v_cache"])
+    kc[L:] = so.round_bf16(so.rope(f64(x["k_new"]), L, cfg.rope_theta))
+    vc[L:] = f64(x["v_new"])
+    q_rot = so.rope(f64(x["q_new"]), L, cfg.rope_theta)
+    rng = np.random.default_rng(0)
+    total = 0.0
+    for s in range(warmup + steps):
+        toks = rng.integers(0, n, size=rows_per_step)
+        t0 = time.perf_counter()
+        for i in toks:
+            so.attend_range(q_rot[i:i + 1], kc, vc, L + int(i), 0, L + int(i) + 1)
+        if s >= warmup:
+            total += time.perf_counter() - t0
+    return total / steps, so.num_threads()
+
+
+def cpu_baseline_full_step(cfg):
+    """One full step of the oracle (all query rows), threads as the oracle uses them."""
+    from oracle import step_oracle as so
+    x = W.make_step_inputs(cfg)
+    f64 = lambda t: np.ascontiguousarray(t.to(torch.float64).numpy())
+    L, n = cfg.cache_len, cfg.num_new
+    kc = np.zeros((L + n, cfg.num_kv_heads, cfg.head_dim))
+    vc = np.zeros_like(kc)
+    kc[:L], vc[:L] = f64(x["k_cache"]), f64(x["v_cache"])
+    q, k, v = f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"])
+    t0 = time.perf_counter()
+    so.step(q, k, v, kc, vc, L, cfg.rope_theta, storage="bf16")
+    dt = time.perf_counter() - t0
+    return dt, so.num_threads()
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return None
+    cfg = W.STEP_7B
+    # attend_range walks one token's query heads serially: one sample = one token x 28 heads
+    probe, threads = oracle_sample_time(cfg, 1, 1, 1)
+    budget_s = 120.0
+    total_steps = args.steps + args.warmup
+    per = max(1, min(cfg.num_new, int(budget_s / max(total_steps, 1) / max(probe, 1e-9))))
+    if probe * total_steps > 2 * budget_s:
+        steps = max(1, int(budget_s / probe) - args.warmup)
+    else:
+        steps = args.steps
+    t_step, threads = oracle_sample_time(cfg, per, steps, min(args.warmup, 3))
+    us_full = t_step / per * cfg.num_new * 1e6
+    line = {
+        "impl": "reference", "metric": "new-frame step-attention latency", "value": round(us_full, 1),
+        "unit": "us/step", "n_gpus": world, "steps": steps, "warmup": min(args.warmup, 3),
+        "ms_per_step": us_full / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: 28q/4kv heads, head_dim 128, L=4096, n=196, theta 1e6 "
+                               "(fp64 CPU oracle of the same step)"},
+        "cpu_baseline": {"value": round(us_full, 1), "unit": "us/step", "cores": 1, "kind": "oracle",
+                         "sample": f"{per} of {cfg.num_new} query tokens (all 28 heads) per step, attention only, "
+                                   f"serial oracle routine; scaled by {cfg.num_new}/{per}"},
+        "e2e": {"value": round(us_full, 1), "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    if steps != args.steps:
+        line["config"]["note"] = f"steps reduced from {args.steps} to {steps} to bound the CPU run"
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=65536)
+    ap.add_argument("--warmup", type=int, default=3200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        line = run_reference(args, rank, world)
+        if line is not None:
+            print(json.dumps(line), flush=True)
+        return
+
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        torch.cuda.set_device(local_rank)
+        dist_mod.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+        dist = dist_mod
+    line = run_ours(args, rank, world, local_rank, dist)
+    if line is not None:
+        if world == 1 and not args.no_cpu_baseline:
+            dt, threads = cpu_baseline_full_step(W.STEP_7B)
+            line["cpu_baseline"] = {
+                "value": round(dt * 1e6, 1), "unit": "us/step", "cores": threads, "kind": "oracle",
+                "sample": "1 full step of the same workload (all 196 tokens x 28 heads), rotate + append + attention",
+            }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,178 @@
+/*
+ * libevln: step attention for KV-cache reuse with contiguous RoPE on NVIDIA B200 (sm_100a).
+ *
+ * One navigation step of the paper's inference scheme (Sec. 3.2, "KV Cache Reuse with
+ * Contiguous RoPE") processes only the newly observed frame: its n tokens receive the
+ * position ids L .. L+n-1 that continue the cached sequence of length L, their queries and
+ * keys are rotated by RoPE at those positions, the rotated keys and the values are appended
+ * to the reused cache, and the n new queries attend causally to all L+n cached tokens
+ * (grouped-query attention).  Per transformer layer this is three calls:
+ *
+ *     evlnRopeAppend  ->  evlnStepAttention  ->  evlnStepCombine
+ *
+ * plus evlnPaged* variants for a batch of episodes whose caches live in a page pool.
+ *
+ * Conventions
+ *  - Every data pointer is DEVICE memory owned by the caller unless its name starts with
+ *    h_ (host memory, read during the call).  The library never allocates or frees in
+ *    these calls and keeps no reference to caller memory after a call returns.
+ *  - All device base pointers must be 16-byte aligned, token strides multiples of 8
+ *    elements (bf16) / 4 elements (f32); otherwise EVLN_INVALID_VALUE.
+ *  - Calls validate on the host, then enqueue kernels on `stream` (a cudaStream_t passed as
+ *    void*; NULL = default stream) and return without synchronising.  Argument errors
+ *    launch nothing.  EVLN_CUDA_ERROR wraps a failed launch; evlnGetLastCudaError gives
+ *    the cudaError_t value.
+ *  - The library does not advance L: the caller passes the pre-step cache length to all
+ *    three calls of a step and adds n afterwards.
+ *  - For fixed parameters the split schedule is fixed, so results are bitwise reproducible.
+ *  - One handle per host thread.  There is no CPU fallback.
+ *
+ * Layouts (D = head_dim, G = num_q_heads / num_kv_heads, query head h uses kv head h / G)
+ *    q_new          [n, Hq, D]   token stride given in elements, head stride D
+ *    k_new, v_new   [n, Hkv, D]  same
+ *    k_cache,v_cache[Hkv, cache_capacity, D]            (contiguous cache, one layer)
+ *    k_pool, v_pool [num_pages, Hkv, page_size, D]      (paged cache, one layer)
+ *    q_rot          [Hkv, n*G, D] row r = i*G + (h % G) (scratch written by RopeAppend)
+ *    out            [n, Hq, D]   contiguous, same dtype as the inputs
+ *    lse_out        [n, Hq]      float, natural-log sum-exp of the scaled logits (optional)
+ */
+#ifndef EVLN_H_
+#define EVLN_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EVLN_OK = 0,
+    EVLN_INVALID_VALUE = 1,      /* null / misaligned pointer, bad shape, bad struct_size      */
+    EVLN_NOT_SUPPORTED = 2,      /* shape or dtype outside what the kernels implement          */
+    EVLN_CACHE_FULL = 3,         /* cache_len + num_new > cache_capacity (or page table short) */
+    EVLN_WORKSPACE_TOO_SMALL = 4,
+    EVLN_CUDA_ERROR = 5,
+    EVLN_DEVICE_TIMEOUT = 6      /* a bounded wait inside a kernel expired (see DeviceStatus)  */
+} evlnStatus_t;
+
+typedef enum { EVLN_BF16 = 0, EVLN_F32 = 1 } evlnDType_t;
+
+/* Attention kernel choice.  AUTO: tensor-core kernel (tcgen05 MMA, TMEM accumulators, TMA
+ * tiles) for bf16 with head_dim 128; the fp32 SIMT kernel otherwise.  SIMT forces the
+ * SIMT kernel (any dtype), which exists for the fp32 precision target and as an
+ * independent on-device cross-check.                                                        */
+typedef enum { EVLN_KERNEL_AUTO = 0, EVLN_KERNEL_SIMT = 1 } evlnKernel_t;
+
+typedef struct evlnContext* evlnHandle_t;
+
+/* One layer, one episode, contiguous cache. */
+typedef struct {
+    size_t struct_size;      /* sizeof(evlnStepParams)                                       */
+    int dtype;               /* evlnDType_t of q/k/v, cache, q_rot and out                   */
+    int num_q_heads;         /* Hq                                                           */
+    int num_kv_heads;        /* Hkv, divides Hq                                              */
+    int head_dim;            /* D: 64 or 128                                                 */
+    int cache_len;           /* L >= 0: tokens already cached (0 = instruction prefill)      */
+    int num_new;             /* n >= 0: new tokens, rotated at positions L .. L+n-1          */
+    int cache_capacity;      /* token slots per kv head in k_cache / v_cache                 */
+    int num_splits;          /* KV splits; 0 = library heuristic                             */
+    int kernel;              /* evlnKernel_t                                                 */
+    float softmax_scale;     /* 0 -> 1/sqrt(D)                                               */
+    double rope_theta;       /* RoPE base, > 0                                               */
+} evlnStepParams;
+
+/* A batch of episodes on a page pool (one layer).  Episode b has h_cache_lens[b] cached
+ * tokens and its new tokens are rows h_new_offsets[b] .. h_new_offsets[b+1]-1 of the packed
+ * q_new/k_new/v_new/out.  Row p of its page table lists pool pages in sequence order and
+ * must already cover cache_len + num_new tokens (the caller hands out pages).              */
+typedef struct {
+    size_t struct_size;      /* sizeof(evlnPagedParams)                                      */
+    int dtype;               /* EVLN_BF16 only                                               */
+    int num_q_heads, num_kv_heads, head_dim;      /* head_dim 128                            */
+    int batch;               /* number of episodes, 1 .. 256                                 */
+    int page_size;           /* tokens per page: 64                                          */
+    int num_pages;           /* pages in the pool                                            */
+    int max_pages_per_seq;   /* row length of d_page_table                                   */
+    int kv_chunk_tiles;      /* max 128-key tiles per work item; 0 = library heuristic       */
+    float softmax_scale;     /* 0 -> 1/sqrt(D)                                               */
+    double rope_theta;
+} evlnPagedParams;
+
+/* ---- handle, errors ------------------------------------------------------------------- */
+
+/* Creates a handle bound to CUDA device `device` (allocates a 4-byte device status word and
+ * resolves the driver's tensor-map encoder).  Sec. 3.2 has no counterpart: plumbing.        */
+evlnStatus_t evlnCreate(evlnHandle_t* handle, int device);
+evlnStatus_t evlnDestroy(evlnHandle_t handle);
+const char* evlnGetErrorString(evlnStatus_t status);
+/* cudaError_t value of the most recent EVLN_CUDA_ERROR on this handle (0 if none). */
+int evlnGetLastCudaError(evlnHandle_t handle);
+/* Synchronises `stream`, reads and clears the device status word.  *device_status = 0 when no
+ * kernel gave up on a bounded wait; otherwise a code identifying the wait that expired and
+ * the function returns EVLN_DEVICE_TIMEOUT (the outputs of that step are then invalid).     */
+evlnStatus_t evlnGetDeviceStatus(evlnHandle_t handle, void* stream, int* device_status);
+
+/* ---- contiguous cache ------------------------------------------------------------------- */
+
+/* Number of KV splits the attention/combine pair will use for these parameters.            */
+evlnStatus_t evlnStepNumSplits(evlnHandle_t handle, const evlnStepParams* params, int* num_splits);
+/* Bytes of `workspace` needed by evlnStepAttention / evlnStepCombine:
+ * num_splits * Hkv * n*G * (D + 1) floats (per-split outputs and log-sum-exps), rounded up. */
+evlnStatus_t evlnStepWorkspaceSize(evlnHandle_t handle, const evlnStepParams* params, size_t* bytes);
+/* Bytes of the q_rot scratch: n * Hq * D elements, rounded up to 256. */
+evlnStatus_t evlnStepQRotSize(evlnHandle_t handle, const evlnStepParams* params, size_t* bytes);
+
+/* Step 1 (Sec. 3.2: contiguous position ids, RoPE, concatenation with the cache).
+ * Rotates the new queries at positions L+i into q_rot (grouped by kv head), rotates the new
+ * keys and stores them, with the values copied bit-exactly, into cache slots L .. L+n-1.
+ * Angles are formed in double precision, products in float (double for EVLN_F32), one
+ * rounding to the storage dtype.  Slots outside L .. L+n-1 are not touched.
+ * Errors: EVLN_CACHE_FULL if L+n > cache_capacity; n = 0 returns EVLN_OK and launches nothing. */
+evlnStatus_t evlnRopeAppend(evlnHandle_t handle, const evlnStepParams* params,
+                            const void* q_new, const void* k_new, const void* v_new,
+                            long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                            void* q_rot, void* k_cache, void* v_cache, void* stream);
+
+/* Step 2 (Sec. 3.2: prefill of the current frame only, against the reused cache).
+ * Causal attention of the n rotated queries over cache slots 0 .. L+n-1 (query i sees slots
+ * 0 .. L+i), split over the keys; writes per-split normalised outputs and log-sum-exps into
+ * `workspace`.  Must run after evlnRopeAppend of the same step on the same stream.          */
+evlnStatus_t evlnStepAttention(evlnHandle_t handle, const evlnStepParams* params,
+                               const void* q_rot, const void* k_cache, const void* v_cache,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/* Step 3: merges the splits, O = sum_s e^{lse_s-M} O_s / sum_s e^{lse_s-M}, M = max_s lse_s,
+ * rounds once to the storage dtype and scatters rows back to [n, Hq, D].  lse_out may be NULL. */
+evlnStatus_t evlnStepCombine(evlnHandle_t handle, const evlnStepParams* params,
+                             const void* workspace, void* out, float* lse_out, void* stream);
+
+/* ---- paged cache, batch of episodes ----------------------------------------------------- */
+
+/* The three calls take the episode lengths from HOST arrays (h_cache_lens [batch],
+ * h_new_offsets [batch+1]); they travel to the kernels as launch parameters, so no copy is
+ * enqueued.  d_page_table is DEVICE memory, int [batch, max_pages_per_seq].                 */
+evlnStatus_t evlnPagedWorkspaceSize(evlnHandle_t handle, const evlnPagedParams* params,
+                                    const int* h_cache_lens, const int* h_new_offsets,
+                                    size_t* bytes);
+/* As evlnRopeAppend, slot of token L_b+i = page_table[b][(L_b+i)/page] * page + (L_b+i)%page.
+ * Additionally zero-fills the value slots after the last appended token up to the end of
+ * its page, so that a partly filled page never exposes stale bits to the attention kernel. */
+evlnStatus_t evlnPagedRopeAppend(evlnHandle_t handle, const evlnPagedParams* params,
+                                 const void* q_new, const void* k_new, const void* v_new,
+                                 const int* h_cache_lens, const int* h_new_offsets,
+                                 const int* d_page_table, void* q_rot, void* k_pool, void* v_pool,
+                                 void* stream);
+evlnStatus_t evlnPagedStepAttention(evlnHandle_t handle, const evlnPagedParams* params,
+                                    const void* q_rot, const void* k_pool, const void* v_pool,
+                                    const int* h_cache_lens, const int* h_new_offsets,
+                                    const int* d_page_table, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+evlnStatus_t evlnPagedStepCombine(evlnHandle_t handle, const evlnPagedParams* params,
+                                  const void* workspace, const int* h_cache_lens,
+                                  const int* h_new_offsets, void* out, float* lse_out,
+                                  void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EVLN_H_ */

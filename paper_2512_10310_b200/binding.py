@@ -1,0 +1,255 @@
+"""ctypes binding of ``libevln.so``: same names as the C entry points, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  PyTorch is used for device memory
+and streams.  There is no fallback: loading fails loudly when the library has not been built
+(``python -c "import __graft_entry__ as g; g.build()"`` or ``build_library()`` below).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from ctypes import (POINTER, Structure, byref, c_char_p, c_double, c_float, c_int, c_long, c_size_t,
+                    c_void_p)
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_PKG)
+LIB_PATH = os.path.join(_PKG, "lib", "libevln.so")
+_SOURCES = ["evln_api.cu", "attn_tcgen05.cuh", "attn_simt.cuh", "combine.cuh", "rope_append.cuh",
+            "common.cuh", "ptx_sm100.cuh"]
+
+EVLN_OK, EVLN_INVALID_VALUE, EVLN_NOT_SUPPORTED, EVLN_CACHE_FULL = 0, 1, 2, 3
+EVLN_WORKSPACE_TOO_SMALL, EVLN_CUDA_ERROR, EVLN_DEVICE_TIMEOUT = 4, 5, 6
+EVLN_BF16, EVLN_F32 = 0, 1
+EVLN_KERNEL_AUTO, EVLN_KERNEL_SIMT = 0, 1
+
+EXPORTS = [
+    "evlnCreate", "evlnDestroy", "evlnGetErrorString", "evlnGetLastCudaError", "evlnGetDeviceStatus",
+    "evlnStepNumSplits", "evlnStepWorkspaceSize", "evlnStepQRotSize",
+    "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine",
+    "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
+]
+
+
+class evlnStepParams(Structure):
+    _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_q_heads", c_int),
+                ("num_kv_heads", c_int), ("head_dim", c_int), ("cache_len", c_int),
+                ("num_new", c_int), ("cache_capacity", c_int), ("num_splits", c_int),
+                ("kernel", c_int), ("softmax_scale", c_float), ("rope_theta", c_double)]
+
+
+class evlnPagedParams(Structure):
+    _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_q_heads", c_int),
+                ("num_kv_heads", c_int), ("head_dim", c_int), ("batch", c_int),
+                ("page_size", c_int), ("num_pages", c_int), ("max_pages_per_seq", c_int),
+                ("kv_chunk_tiles", c_int), ("softmax_scale", c_float), ("rope_theta", c_double)]
+
+
+class EvlnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {error_string(status)} ({status})")
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compile the CUDA sources into ``lib/libevln.so`` for sm_100a (in-tree)."""
+    src_dir = os.path.join(_PKG, "csrc")
+    srcs = [os.path.join(src_dir, s) for s in _SOURCES] + [os.path.join(_ROOT, "include", "evln.h")]
+    if not force and os.path.exists(LIB_PATH) and all(
+            os.path.getmtime(LIB_PATH) >= os.path.getmtime(s) for s in srcs):
+        return LIB_PATH
+    os.makedirs(os.path.dirname(LIB_PATH), exist_ok=True)
+    tmp = LIB_PATH + f".tmp{os.getpid()}"
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-o", tmp, os.path.join(src_dir, "evln_api.cu")]
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
+    return LIB_PATH
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library; raises if it has not been built (no fallback of any kind)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with __graft_entry__.build() "
+                              "(nvcc, sm_100a); there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        L.evlnGetErrorString.restype = c_char_p
+        L.evlnGetErrorString.argtypes = [c_int]
+        L.evlnCreate.argtypes = [POINTER(c_void_p), c_int]
+        L.evlnDestroy.argtypes = [c_void_p]
+        L.evlnGetLastCudaError.argtypes = [c_void_p]
+        L.evlnGetDeviceStatus.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
+        pp = POINTER(evlnStepParams)
+        L.evlnStepNumSplits.argtypes = [c_void_p, pp, POINTER(c_int)]
+        L.evlnStepWorkspaceSize.argtypes = [c_void_p, pp, POINTER(c_size_t)]
+        L.evlnStepQRotSize.argtypes = [c_void_p, pp, POINTER(c_size_t)]
+        L.evlnRopeAppend.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_long, c_long, c_long,
+                                     c_void_p, c_void_p, c_void_p, c_void_p]
+        L.evlnStepAttention.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
+                                        c_void_p]
+        L.evlnStepCombine.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_void_p]
+        gp = POINTER(evlnPagedParams)
+        ip = POINTER(c_int)
+        L.evlnPagedWorkspaceSize.argtypes = [c_void_p, gp, ip, ip, POINTER(c_size_t)]
+        L.evlnPagedRopeAppend.argtypes = [c_void_p, gp, c_void_p, c_void_p, c_void_p, ip, ip, c_void_p,
+                                          c_void_p, c_void_p, c_void_p, c_void_p]
+        L.evlnPagedStepAttention.argtypes = [c_void_p, gp, c_void_p, c_void_p, c_void_p, ip, ip, c_void_p,
+                                             c_void_p, c_size_t, c_void_p]
+        L.evlnPagedStepCombine.argtypes = [c_void_p, gp, c_void_p, ip, ip, c_void_p, c_void_p, c_void_p]
+        for name in EXPORTS:
+            if name != "evlnGetErrorString":
+                getattr(L, name).restype = c_int
+        _lib = L
+    return _lib
+
+
+def error_string(status: int) -> str:
+    return lib().evlnGetErrorString(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != EVLN_OK:
+        raise EvlnError(status, where)
+
+
+def _ptr(t):
+    """Device (or host) address of a tensor, None -> NULL; raw ints pass through."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return c_void_p(t)
+    return c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return c_void_p(stream)
+    return c_void_p(stream.cuda_stream)
+
+
+def _ints(seq):
+    arr = (c_int * len(seq))(*[int(v) for v in seq])
+    return arr
+
+
+def step_params(dtype, num_q_heads, num_kv_heads, head_dim, cache_len, num_new, cache_capacity,
+                rope_theta, softmax_scale=0.0, num_splits=0, kernel=EVLN_KERNEL_AUTO) -> evlnStepParams:
+    code = {"bf16": EVLN_BF16, "f32": EVLN_F32}.get(dtype, dtype)
+    return evlnStepParams(ctypes.sizeof(evlnStepParams), code, num_q_heads, num_kv_heads, head_dim,
+                          cache_len, num_new, cache_capacity, num_splits, kernel, softmax_scale, rope_theta)
+
+
+def paged_params(num_q_heads, num_kv_heads, head_dim, batch, page_size, num_pages, max_pages_per_seq,
+                 rope_theta, softmax_scale=0.0, kv_chunk_tiles=0, dtype=EVLN_BF16) -> evlnPagedParams:
+    return evlnPagedParams(ctypes.sizeof(evlnPagedParams), dtype, num_q_heads, num_kv_heads, head_dim,
+                           batch, page_size, num_pages, max_pages_per_seq, kv_chunk_tiles, softmax_scale,
+                           rope_theta)
+
+
+# ---- the entry points, by their C names ----------------------------------------------------
+
+def evlnCreate(device: int = 0):
+    h = c_void_p()
+    _check(lib().evlnCreate(byref(h), int(device)), "evlnCreate")
+    return h
+
+
+def evlnDestroy(handle):
+    _check(lib().evlnDestroy(handle), "evlnDestroy")
+
+
+def evlnGetLastCudaError(handle) -> int:
+    return int(lib().evlnGetLastCudaError(handle))
+
+
+def evlnGetDeviceStatus(handle, stream=None) -> int:
+    """Synchronises the stream; returns the device status word (0 = no bounded wait expired)."""
+    v = c_int(0)
+    st = lib().evlnGetDeviceStatus(handle, _stream(stream), byref(v))
+    if st not in (EVLN_OK, EVLN_DEVICE_TIMEOUT):
+        raise EvlnError(st, "evlnGetDeviceStatus")
+    return int(v.value)
+
+
+def evlnStepNumSplits(handle, params) -> int:
+    v = c_int(0)
+    _check(lib().evlnStepNumSplits(handle, byref(params), byref(v)), "evlnStepNumSplits")
+    return int(v.value)
+
+
+def evlnStepWorkspaceSize(handle, params) -> int:
+    v = c_size_t(0)
+    _check(lib().evlnStepWorkspaceSize(handle, byref(params), byref(v)), "evlnStepWorkspaceSize")
+    return int(v.value)
+
+
+def evlnStepQRotSize(handle, params) -> int:
+    v = c_size_t(0)
+    _check(lib().evlnStepQRotSize(handle, byref(params), byref(v)), "evlnStepQRotSize")
+    return int(v.value)
+
+
+def evlnRopeAppend(handle, params, q_new, k_new, v_new, q_rot, k_cache, v_cache, stream=None,
+                   strides=None):
+    """q_new/k_new/v_new: [n,H,D] tensors (last two dims contiguous) or raw addresses + strides."""
+    if strides is None:
+        strides = (q_new.stride(0), k_new.stride(0), v_new.stride(0))
+    _check(lib().evlnRopeAppend(handle, byref(params), _ptr(q_new), _ptr(k_new), _ptr(v_new),
+                                int(strides[0]), int(strides[1]), int(strides[2]), _ptr(q_rot),
+                                _ptr(k_cache), _ptr(v_cache), _stream(stream)), "evlnRopeAppend")
+
+
+def evlnStepAttention(handle, params, q_rot, k_cache, v_cache, workspace, workspace_bytes=None,
+                      stream=None):
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().evlnStepAttention(handle, byref(params), _ptr(q_rot), _ptr(k_cache), _ptr(v_cache),
+                                   _ptr(workspace), int(workspace_bytes), _stream(stream)),
+           "evlnStepAttention")
+
+
+def evlnStepCombine(handle, params, workspace, out, lse_out=None, stream=None):
+    _check(lib().evlnStepCombine(handle, byref(params), _ptr(workspace), _ptr(out), _ptr(lse_out),
+                                 _stream(stream)), "evlnStepCombine")
+
+
+def evlnPagedWorkspaceSize(handle, params, cache_lens, new_offsets) -> int:
+    v = c_size_t(0)
+    _check(lib().evlnPagedWorkspaceSize(handle, byref(params), _ints(cache_lens), _ints(new_offsets),
+                                        byref(v)), "evlnPagedWorkspaceSize")
+    return int(v.value)
+
+
+def evlnPagedRopeAppend(handle, params, q_new, k_new, v_new, cache_lens, new_offsets, page_table,
+                        q_rot, k_pool, v_pool, stream=None):
+    _check(lib().evlnPagedRopeAppend(handle, byref(params), _ptr(q_new), _ptr(k_new), _ptr(v_new),
+                                     _ints(cache_lens), _ints(new_offsets), _ptr(page_table),
+                                     _ptr(q_rot), _ptr(k_pool), _ptr(v_pool), _stream(stream)),
+           "evlnPagedRopeAppend")
+
+
+def evlnPagedStepAttention(handle, params, q_rot, k_pool, v_pool, cache_lens, new_offsets, page_table,
+                           workspace, workspace_bytes=None, stream=None):
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().evlnPagedStepAttention(handle, byref(params), _ptr(q_rot), _ptr(k_pool), _ptr(v_pool),
+                                        _ints(cache_lens), _ints(new_offsets), _ptr(page_table),
+                                        _ptr(workspace), int(workspace_bytes), _stream(stream)),
+           "evlnPagedStepAttention")
+
+
+def evlnPagedStepCombine(handle, params, workspace, cache_lens, new_offsets, out, lse_out=None,
+                         stream=None):
+    _check(lib().evlnPagedStepCombine(handle, byref(params), _ptr(workspace), _ints(cache_lens),
+                                      _ints(new_offsets), _ptr(out), _ptr(lse_out), _stream(stream)),
+           "evlnPagedStepCombine")

@@ -1,0 +1,93 @@
+// Split-reduction combine kernel: merges the per-split partial outputs of the step attention.
+//
+//   M = max_s lse_s,  w_s = e^{lse_s - M},  O = sum_s w_s O_s / sum_s w_s,  lse = M + log sum_s w_s
+//
+// One warp per packed query row: lane s holds lse_s (at most 32 splits), the maximum and the
+// weight sum are warp-shuffle reductions, then each lane merges D/32 contiguous channels with
+// vector loads.  The row is rounded once to the storage dtype and written to its place in the
+// token-major [n, Hq, D] output.  HBM/L2-bound: S*(D+1) floats in, D elements out per row.
+#pragma once
+
+#include "common.cuh"
+
+namespace evln {
+
+struct CombineArgs {
+    const float* o_part;     // [S, Hkv, R, D]
+    const float* lse_part;   // [S, Hkv, R]
+    void* out;               // [n, Hq, D]
+    float* lse_out;          // [n, Hq] or null
+    int Hkv, G, D;
+    int rows;                // R = (total) new tokens * G
+    int num_splits;          // contiguous: S for every row
+    // paged: per-episode split counts are derived from the lengths
+    int batch, unit_rows, chunk_tiles;
+};
+
+template <typename T, int D, bool PAGED, typename LensT>
+__global__ void __launch_bounds__(128)
+combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
+{
+    constexpr int C = D / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long row = (long)blockIdx.x * 4 + warp;      // packed row within kv head
+    const int g = blockIdx.y;
+    if (row >= a.rows) return;
+
+    int S = a.num_splits;
+    if (PAGED) {
+        const int tok = (int)(row / a.G);
+        int lo = 0, hi = a.batch;
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (lens.new_off[mid] <= tok) lo = mid; else hi = mid;
+        }
+        const int b = lo;
+        const int n_b = lens.new_off[b + 1] - lens.new_off[b];
+        const int local_row = (int)(row - (long)lens.new_off[b] * a.G);
+        const int unit = local_row / a.unit_rows;
+        S = ceil_div(unit_kv_tiles(lens.cache_len[b], n_b, a.G, unit, a.unit_rows), a.chunk_tiles);
+    }
+
+    const long stride_s = (long)a.Hkv * a.rows;           // rows between consecutive splits
+    const long prow0 = (long)g * a.rows + row;
+
+    float my_lse = (lane < S) ? a.lse_part[prow0 + lane * stride_s] : -INFINITY;
+    float M = my_lse;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    float w = (my_lse == -INFINITY) ? 0.f : expf(my_lse - M);    // M = -inf only if all are
+    float wsum = w;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, off);
+
+    float acc[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) acc[c] = 0.f;
+    for (int s = 0; s < S; ++s) {
+        const float ws = __shfl_sync(0xffffffffu, w, s);
+        if (ws == 0.f) continue;                               // uniform across the warp
+        const float* op = a.o_part + (prow0 + s * stride_s) * D + lane * C;
+        float v[C];
+        if (C == 4) {
+            float4 x = *reinterpret_cast<const float4*>(op);
+            v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+        } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) v[c] = op[c];
+        }
+#pragma unroll
+        for (int c = 0; c < C; ++c) acc[c] = fmaf(ws, v[c], acc[c]);
+    }
+    const float inv = (wsum > 0.f) ? 1.f / wsum : 0.f;
+
+    const long tok = row / a.G;
+    const int h = g * a.G + (int)(row % a.G);
+    const int Hq = a.Hkv * a.G;
+    T* dst = (T*)a.out + (tok * Hq + h) * D + lane * C;
+#pragma unroll
+    for (int c = 0; c < C; ++c) from_float(acc[c] * inv, dst[c]);
+    if (a.lse_out && lane == 0) a.lse_out[tok * Hq + h] = (wsum > 0.f) ? M + logf(wsum) : -INFINITY;
+}
+
+}  // namespace evln

@@ -1,0 +1,60 @@
+// Shared host/device declarations of libevln's kernels (internal; the public contract is
+// include/evln.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace evln {
+
+constexpr int kMaxBatch = 256;     // paged calls carry per-episode lengths as launch parameters
+constexpr int kMaxSplits = 32;     // a warp merges one split per lane
+constexpr int kTileM = 128;        // query rows per MMA tile
+constexpr int kTileN = 128;        // keys per KV tile
+constexpr int kUnitRows = 2 * kTileM;  // one CTA of the tensor-core kernel owns two query tiles
+
+// Device status codes written by kernels whose bounded waits expire.
+enum DeviceStatus : int {
+    kDevOk = 0,
+    kDevTimeoutProducer = 1,   // TMA producer waiting for a free K/V stage
+    kDevTimeoutMmaQ = 2,       // MMA warp waiting for the Q tiles
+    kDevTimeoutMmaKV = 3,      // MMA warp waiting for a K/V tile
+    kDevTimeoutMmaP = 4,       // MMA warp waiting for the softmax warps' P tile
+    kDevTimeoutSoftmaxS = 5,   // softmax warps waiting for S
+    kDevTimeoutSoftmaxO = 6,   // softmax warps waiting for the final O
+};
+
+// Per-episode lengths of a paged batch, passed by value.
+struct BatchLens {
+    int cache_len[kMaxBatch];
+    int new_off[kMaxBatch + 1];
+};
+
+template <typename T> struct VecTraits;
+template <> struct VecTraits<__nv_bfloat16> { static constexpr int kVec = 8; };
+template <> struct VecTraits<float> { static constexpr int kVec = 4; };
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void from_float(float x, float& y) { y = x; }
+__device__ __forceinline__ void from_float(float x, __nv_bfloat16& y) { y = __float2bfloat16_rn(x); }
+
+// Number of 128-key tiles the rows of unit u (rows [u*unit_rows, ...)) of an episode need.
+__host__ __device__ inline int unit_kv_tiles(int L, int n, int G, int unit, int unit_rows)
+{
+    long last_row = (long)(unit + 1) * unit_rows - 1;
+    long last_tok = last_row / G;
+    if (last_tok > n - 1) last_tok = n - 1;
+    return (int)((L + last_tok + 1 + kTileN - 1) / kTileN);
+}
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Stub lengths for the kernels that serve one episode.
+struct NoLens {
+    int cache_len[1];
+    int new_off[2];
+};
+
+}  // namespace evln

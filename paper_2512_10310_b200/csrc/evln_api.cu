@@ -1,0 +1,546 @@
+// C-ABI entry points of libevln (contract: include/evln.h).  Host-side validation, the split
+// schedule, tensor-map encoding and kernel launches; no allocation in the per-step calls.
+#include "../../include/evln.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <new>
+
+#include "attn_simt.cuh"
+#include "attn_tcgen05.cuh"
+#include "combine.cuh"
+#include "common.cuh"
+#include "rope_append.cuh"
+
+using namespace evln;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct evlnContext {
+    int device;
+    int num_sms;
+    int last_cuda_error;
+    int* d_status;
+    EncodeTiledFn encode;
+};
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int elem_bytes(int dtype) { return dtype == EVLN_BF16 ? 2 : 4; }
+
+evlnStatus_t cuda_fail(evlnHandle_t h, cudaError_t e)
+{
+    h->last_cuda_error = (int)e;
+    return EVLN_CUDA_ERROR;
+}
+
+evlnStatus_t check_step_params(evlnHandle_t h, const evlnStepParams* p)
+{
+    if (!h || !p) return EVLN_INVALID_VALUE;
+    if (p->struct_size != sizeof(evlnStepParams)) return EVLN_INVALID_VALUE;
+    if (p->dtype != EVLN_BF16 && p->dtype != EVLN_F32) return EVLN_INVALID_VALUE;
+    if (p->num_q_heads <= 0 || p->num_kv_heads <= 0 || p->num_q_heads % p->num_kv_heads != 0)
+        return EVLN_INVALID_VALUE;
+    if (p->cache_len < 0 || p->num_new < 0 || p->cache_capacity < 0) return EVLN_INVALID_VALUE;
+    if (!(p->rope_theta > 0.0) || !(p->softmax_scale >= 0.f)) return EVLN_INVALID_VALUE;
+    if (p->num_splits < 0 || p->num_splits > kMaxSplits) return EVLN_INVALID_VALUE;
+    if (p->kernel != EVLN_KERNEL_AUTO && p->kernel != EVLN_KERNEL_SIMT) return EVLN_INVALID_VALUE;
+    if (p->head_dim != 64 && p->head_dim != 128) return EVLN_NOT_SUPPORTED;
+    if ((long)p->cache_len + p->num_new > (long)p->cache_capacity) return EVLN_CACHE_FULL;
+    if ((long)p->num_new * p->num_q_heads / p->num_kv_heads > (1 << 24)) return EVLN_NOT_SUPPORTED;
+    return EVLN_OK;
+}
+
+inline bool use_tensor_kernel(const evlnStepParams* p)
+{
+    return p->kernel == EVLN_KERNEL_AUTO && p->dtype == EVLN_BF16 && p->head_dim == 128;
+}
+
+// Cost model of the split-KV schedule of the tensor-core kernel: `ctas` CTAs run in waves of
+// one per SM, each walks ceil(nkv / S) KV tiles plus a fixed prologue/epilogue; every extra
+// split adds combine traffic.
+int choose_splits_tc(int units_total, int nkv_max, int nkv_min, int num_sms)
+{
+    int best = 1;
+    double best_cost = 1e30;
+    const int smax = nkv_min < kMaxSplits ? (nkv_min < 1 ? 1 : nkv_min) : kMaxSplits;
+    for (int s = 1; s <= smax; ++s) {
+        const double waves = ceil((double)units_total * s / num_sms);
+        const double cost = waves * (ceil((double)nkv_max / s) + 2.0) + 0.3 * s;
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
+int resolve_splits(evlnHandle_t h, const evlnStepParams* p)
+{
+    if (p->num_new == 0) return 1;
+    if (p->num_splits > 0) return p->num_splits;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const int R = p->num_new * G;
+    const int T = p->cache_len + p->num_new;
+    if (use_tensor_kernel(p)) {
+        const int units = ceil_div(R, kUnitRows);
+        const int nkv_max = unit_kv_tiles(p->cache_len, p->num_new, G, units - 1, kUnitRows);
+        const int nkv_min = unit_kv_tiles(p->cache_len, p->num_new, G, 0, kUnitRows);
+        return choose_splits_tc(units * p->num_kv_heads, nkv_max, nkv_min, h->num_sms);
+    }
+    const int blocks = ceil_div(R, 4) * p->num_kv_heads;
+    int s = ceil_div(2 * h->num_sms, blocks);
+    const int cap = ceil_div(T, 64);
+    if (s > cap) s = cap;
+    if (s > kMaxSplits) s = kMaxSplits;
+    if (s < 1) s = 1;
+    return s;
+}
+
+size_t partial_bytes(int splits, int Hkv, long rows, int D)
+{
+    return round_up((size_t)splits * Hkv * rows * (D + 1) * sizeof(float), 256);
+}
+
+bool encode_map(evlnHandle_t h, CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,
+                const cuuint64_t* strides_bytes, const cuuint32_t* box)
+{
+    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base),
+                           dims, strides_bytes, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+evlnStatus_t check_paged_params(evlnHandle_t h, const evlnPagedParams* p, const int* lens, const int* offs)
+{
+    if (!h || !p || !lens || !offs) return EVLN_INVALID_VALUE;
+    if (p->struct_size != sizeof(evlnPagedParams)) return EVLN_INVALID_VALUE;
+    if (p->num_q_heads <= 0 || p->num_kv_heads <= 0 || p->num_q_heads % p->num_kv_heads != 0)
+        return EVLN_INVALID_VALUE;
+    if (p->batch < 1 || p->num_pages < 1 || p->max_pages_per_seq < 1 || p->kv_chunk_tiles < 0)
+        return EVLN_INVALID_VALUE;
+    if (!(p->rope_theta > 0.0) || !(p->softmax_scale >= 0.f)) return EVLN_INVALID_VALUE;
+    if (p->dtype != EVLN_BF16 || p->head_dim != 128 || p->page_size != 64 || p->batch > kMaxBatch)
+        return EVLN_NOT_SUPPORTED;
+    if (offs[0] != 0) return EVLN_INVALID_VALUE;
+    for (int b = 0; b < p->batch; ++b) {
+        if (lens[b] < 0 || offs[b + 1] < offs[b]) return EVLN_INVALID_VALUE;
+        const long tokens = (long)lens[b] + (offs[b + 1] - offs[b]);
+        if ((tokens + p->page_size - 1) / p->page_size > p->max_pages_per_seq) return EVLN_CACHE_FULL;
+    }
+    if ((long)offs[p->batch] * p->num_q_heads / p->num_kv_heads > (1 << 24)) return EVLN_NOT_SUPPORTED;
+    return EVLN_OK;
+}
+
+// Work-item size (KV tiles) and the largest split count of a paged batch.
+void paged_schedule(evlnHandle_t h, const evlnPagedParams* p, const int* lens, const int* offs,
+                    int* chunk_tiles, int* max_splits, long* items)
+{
+    const int G = p->num_q_heads / p->num_kv_heads;
+    long total = 0;
+    int nkv_max = 1;
+    for (int b = 0; b < p->batch; ++b) {
+        const int n = offs[b + 1] - offs[b];
+        const int units = ceil_div(n * G, kUnitRows);
+        for (int u = 0; u < units; ++u) {
+            const int nkv = unit_kv_tiles(lens[b], n, G, u, kUnitRows);
+            total += nkv;
+            if (nkv > nkv_max) nkv_max = nkv;
+        }
+    }
+    total *= p->num_kv_heads;
+    int chunk = p->kv_chunk_tiles;
+    if (chunk <= 0) {
+        chunk = (int)((total + (long)h->num_sms * 4 - 1) / ((long)h->num_sms * 4));
+        if (chunk < 8) chunk = 8;
+    }
+    if (chunk < ceil_div(nkv_max, kMaxSplits)) chunk = ceil_div(nkv_max, kMaxSplits);
+    long cnt = 0;
+    for (int b = 0; b < p->batch; ++b) {
+        const int n = offs[b + 1] - offs[b];
+        const int units = ceil_div(n * G, kUnitRows);
+        for (int u = 0; u < units; ++u) cnt += ceil_div(unit_kv_tiles(lens[b], n, G, u, kUnitRows), chunk);
+    }
+    *chunk_tiles = chunk;
+    *max_splits = ceil_div(nkv_max, chunk);
+    *items = cnt * p->num_kv_heads;
+}
+
+void fill_lens(BatchLens* bl, const evlnPagedParams* p, const int* lens, const int* offs)
+{
+    memset(bl, 0, sizeof(*bl));
+    for (int b = 0; b < p->batch; ++b) bl->cache_len[b] = lens[b];
+    for (int b = 0; b <= p->batch; ++b) bl->new_off[b] = offs[b];
+}
+
+template <typename T>
+evlnStatus_t launch_combine(evlnHandle_t h, const CombineArgs& a, int D, bool paged, const BatchLens* bl,
+                            cudaStream_t st)
+{
+    dim3 grid(ceil_div(a.rows, 4), a.Hkv);
+    if (paged) {
+        if (D == 128) combine_kernel<T, 128, true, BatchLens><<<grid, 128, 0, st>>>(a, *bl);
+        else return EVLN_NOT_SUPPORTED;
+    } else {
+        NoLens nl = {};
+        if (D == 128) combine_kernel<T, 128, false, NoLens><<<grid, 128, 0, st>>>(a, nl);
+        else combine_kernel<T, 64, false, NoLens><<<grid, 128, 0, st>>>(a, nl);
+    }
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* evlnGetErrorString(evlnStatus_t s)
+{
+    switch (s) {
+        case EVLN_OK: return "EVLN_OK";
+        case EVLN_INVALID_VALUE: return "EVLN_INVALID_VALUE";
+        case EVLN_NOT_SUPPORTED: return "EVLN_NOT_SUPPORTED";
+        case EVLN_CACHE_FULL: return "EVLN_CACHE_FULL";
+        case EVLN_WORKSPACE_TOO_SMALL: return "EVLN_WORKSPACE_TOO_SMALL";
+        case EVLN_CUDA_ERROR: return "EVLN_CUDA_ERROR";
+        case EVLN_DEVICE_TIMEOUT: return "EVLN_DEVICE_TIMEOUT";
+    }
+    return "EVLN_UNKNOWN_STATUS";
+}
+
+evlnStatus_t evlnCreate(evlnHandle_t* handle, int device)
+{
+    if (!handle) return EVLN_INVALID_VALUE;
+    *handle = nullptr;
+    evlnContext* h = new (std::nothrow) evlnContext();
+    if (!h) return EVLN_CUDA_ERROR;
+    h->device = device;
+    h->last_cuda_error = 0;
+    h->d_status = nullptr;
+    h->encode = nullptr;
+    cudaError_t e = cudaSetDevice(device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) { delete h; return EVLN_CUDA_ERROR; }
+    if (prop.major != 10) { delete h; return EVLN_NOT_SUPPORTED; }
+    h->num_sms = prop.multiProcessorCount;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) { delete h; return EVLN_CUDA_ERROR; }
+    h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    e = cudaMalloc(&h->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_tc_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kTcSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_tc_kernel<true, BatchLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kTcSmemBytes);
+    if (e != cudaSuccess) {
+        if (h->d_status) cudaFree(h->d_status);
+        delete h;
+        return EVLN_CUDA_ERROR;
+    }
+    *handle = h;
+    return EVLN_OK;
+}
+
+evlnStatus_t evlnDestroy(evlnHandle_t h)
+{
+    if (!h) return EVLN_INVALID_VALUE;
+    if (h->d_status) cudaFree(h->d_status);
+    delete h;
+    return EVLN_OK;
+}
+
+int evlnGetLastCudaError(evlnHandle_t h) { return h ? h->last_cuda_error : 0; }
+
+evlnStatus_t evlnGetDeviceStatus(evlnHandle_t h, void* stream, int* device_status)
+{
+    if (!h || !device_status) return EVLN_INVALID_VALUE;
+    cudaStream_t st = (cudaStream_t)stream;
+    int v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e == cudaSuccess && v != 0) e = cudaMemsetAsync(h->d_status, 0, sizeof(int), st);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    *device_status = v;
+    return v == 0 ? EVLN_OK : EVLN_DEVICE_TIMEOUT;
+}
+
+evlnStatus_t evlnStepNumSplits(evlnHandle_t h, const evlnStepParams* p, int* num_splits)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (!num_splits) return EVLN_INVALID_VALUE;
+    *num_splits = resolve_splits(h, p);
+    return EVLN_OK;
+}
+
+evlnStatus_t evlnStepWorkspaceSize(evlnHandle_t h, const evlnStepParams* p, size_t* bytes)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (!bytes) return EVLN_INVALID_VALUE;
+    const long rows = (long)p->num_new * (p->num_q_heads / p->num_kv_heads);
+    *bytes = partial_bytes(resolve_splits(h, p), p->num_kv_heads, rows, p->head_dim);
+    return EVLN_OK;
+}
+
+evlnStatus_t evlnStepQRotSize(evlnHandle_t h, const evlnStepParams* p, size_t* bytes)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (!bytes) return EVLN_INVALID_VALUE;
+    *bytes = round_up((size_t)p->num_new * p->num_q_heads * p->head_dim * elem_bytes(p->dtype), 256);
+    return EVLN_OK;
+}
+
+evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
+                            const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                            void* q_rot, void* k_cache, void* v_cache, void* stream)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (p->num_new == 0) return EVLN_OK;
+    if (!q_new || !k_new || !v_new || !q_rot || !k_cache || !v_cache) return EVLN_INVALID_VALUE;
+    if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(q_rot) ||
+        !aligned16(k_cache) || !aligned16(v_cache))
+        return EVLN_INVALID_VALUE;
+    const int vec = 16 / elem_bytes(p->dtype);
+    if (q_stride_tok < (long)p->num_q_heads * p->head_dim || k_stride_tok < (long)p->num_kv_heads * p->head_dim ||
+        v_stride_tok < (long)p->num_kv_heads * p->head_dim)
+        return EVLN_INVALID_VALUE;
+    if (q_stride_tok % vec || k_stride_tok % vec || v_stride_tok % vec) return EVLN_INVALID_VALUE;
+
+    RopeArgs a = {};
+    a.q_new = q_new; a.k_new = k_new; a.v_new = v_new;
+    a.q_rot = q_rot; a.k_cache = k_cache; a.v_cache = v_cache;
+    a.page_table = nullptr;
+    a.q_stride = q_stride_tok; a.k_stride = k_stride_tok; a.v_stride = v_stride_tok;
+    a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.cache_len = p->cache_len; a.num_new = p->num_new; a.cache_cap = p->cache_capacity;
+    a.log2_theta = log2(p->rope_theta);
+    NoLens nl = {};
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->dtype == EVLN_BF16)
+        rope_append_kernel<__nv_bfloat16, false, NoLens><<<p->num_new, 256, 0, st>>>(a, nl);
+    else
+        rope_append_kernel<float, false, NoLens><<<p->num_new, 256, 0, st>>>(a, nl);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const void* q_rot, const void* k_cache,
+                               const void* v_cache, void* workspace, size_t workspace_bytes, void* stream)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (p->num_new == 0) return EVLN_OK;
+    if (!q_rot || !k_cache || !v_cache || !workspace) return EVLN_INVALID_VALUE;
+    if (!aligned16(q_rot) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(workspace))
+        return EVLN_INVALID_VALUE;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const int R = p->num_new * G;
+    const int D = p->head_dim;
+    const int S = resolve_splits(h, p);
+    if (workspace_bytes < partial_bytes(S, p->num_kv_heads, R, D)) return EVLN_WORKSPACE_TOO_SMALL;
+    float* o_part = (float*)workspace;
+    float* lse_part = o_part + (size_t)S * p->num_kv_heads * R * D;
+    const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = (cudaStream_t)stream;
+
+    if (use_tensor_kernel(p)) {
+        const int T = p->cache_len + p->num_new;
+        CUtensorMap tm_q, tm_k, tm_v;
+        {
+            cuuint64_t dims[3] = {128, (cuuint64_t)R, (cuuint64_t)p->num_kv_heads};
+            cuuint64_t strides[2] = {256, (cuuint64_t)R * 256};
+            cuuint32_t box[3] = {64, 128, 1};
+            if (!encode_map(h, &tm_q, q_rot, 3, dims, strides, box)) return EVLN_INVALID_VALUE;
+        }
+        {
+            // rows past L+n read as zeros, so stale slots never reach the tensor core
+            cuuint64_t dims[3] = {128, (cuuint64_t)T, (cuuint64_t)p->num_kv_heads};
+            cuuint64_t strides[2] = {256, (cuuint64_t)p->cache_capacity * 256};
+            cuuint32_t box[3] = {64, 128, 1};
+            if (!encode_map(h, &tm_k, k_cache, 3, dims, strides, box)) return EVLN_INVALID_VALUE;
+            if (!encode_map(h, &tm_v, v_cache, 3, dims, strides, box)) return EVLN_INVALID_VALUE;
+        }
+        TcAttnArgs a = {};
+        a.o_part = o_part; a.lse_part = lse_part; a.page_table = nullptr; a.status = h->d_status;
+        a.Hkv = p->num_kv_heads; a.G = G; a.rows = R;
+        a.cache_len = p->cache_len; a.num_new = p->num_new; a.num_splits = S;
+        a.units_per_head = ceil_div(R, kUnitRows);
+        a.scale_log2 = scale * 1.4426950408889634f;
+        NoLens nl = {};
+        const int grid = S * p->num_kv_heads * a.units_per_head;
+        attn_tc_kernel<false, NoLens><<<grid, kTcThreads, kTcSmemBytes, st>>>(tm_q, tm_k, tm_v, a, nl);
+    } else {
+        SimtAttnArgs a = {};
+        a.q_rot = q_rot; a.k_cache = k_cache; a.v_cache = v_cache;
+        a.o_part = o_part; a.lse_part = lse_part;
+        a.Hkv = p->num_kv_heads; a.G = G; a.D = D;
+        a.cache_len = p->cache_len; a.num_new = p->num_new; a.cache_cap = p->cache_capacity;
+        a.num_splits = S; a.scale = scale;
+        dim3 grid(ceil_div(R, 4), p->num_kv_heads, S);
+        if (p->dtype == EVLN_BF16) {
+            if (D == 128) attn_simt_kernel<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(a);
+            else attn_simt_kernel<__nv_bfloat16, 64><<<grid, 128, 0, st>>>(a);
+        } else {
+            if (D == 128) attn_simt_kernel<float, 128><<<grid, 128, 0, st>>>(a);
+            else attn_simt_kernel<float, 64><<<grid, 128, 0, st>>>(a);
+        }
+    }
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void* workspace, void* out,
+                             float* lse_out, void* stream)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (p->num_new == 0) return EVLN_OK;
+    if (!workspace || !out || !aligned16(workspace) || !aligned16(out)) return EVLN_INVALID_VALUE;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const int R = p->num_new * G;
+    const int S = resolve_splits(h, p);
+    CombineArgs a = {};
+    a.o_part = (const float*)workspace;
+    a.lse_part = a.o_part + (size_t)S * p->num_kv_heads * R * p->head_dim;
+    a.out = out; a.lse_out = lse_out;
+    a.Hkv = p->num_kv_heads; a.G = G; a.D = p->head_dim; a.rows = R; a.num_splits = S;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->dtype == EVLN_BF16) return launch_combine<__nv_bfloat16>(h, a, p->head_dim, false, nullptr, st);
+    return launch_combine<float>(h, a, p->head_dim, false, nullptr, st);
+}
+
+// ---- paged -------------------------------------------------------------------------------
+
+evlnStatus_t evlnPagedWorkspaceSize(evlnHandle_t h, const evlnPagedParams* p, const int* h_cache_lens,
+                                    const int* h_new_offsets, size_t* bytes)
+{
+    evlnStatus_t s = check_paged_params(h, p, h_cache_lens, h_new_offsets);
+    if (s != EVLN_OK) return s;
+    if (!bytes) return EVLN_INVALID_VALUE;
+    int chunk, smax;
+    long items;
+    paged_schedule(h, p, h_cache_lens, h_new_offsets, &chunk, &smax, &items);
+    const long rows = (long)h_new_offsets[p->batch] * (p->num_q_heads / p->num_kv_heads);
+    *bytes = partial_bytes(smax, p->num_kv_heads, rows, p->head_dim);
+    return EVLN_OK;
+}
+
+evlnStatus_t evlnPagedRopeAppend(evlnHandle_t h, const evlnPagedParams* p, const void* q_new, const void* k_new,
+                                 const void* v_new, const int* h_cache_lens, const int* h_new_offsets,
+                                 const int* d_page_table, void* q_rot, void* k_pool, void* v_pool, void* stream)
+{
+    evlnStatus_t s = check_paged_params(h, p, h_cache_lens, h_new_offsets);
+    if (s != EVLN_OK) return s;
+    const int total = h_new_offsets[p->batch];
+    if (total == 0) return EVLN_OK;
+    if (!q_new || !k_new || !v_new || !d_page_table || !q_rot || !k_pool || !v_pool) return EVLN_INVALID_VALUE;
+    if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(q_rot) ||
+        !aligned16(k_pool) || !aligned16(v_pool))
+        return EVLN_INVALID_VALUE;
+    RopeArgs a = {};
+    a.q_new = q_new; a.k_new = k_new; a.v_new = v_new;
+    a.q_rot = q_rot; a.k_cache = k_pool; a.v_cache = v_pool; a.page_table = d_page_table;
+    a.q_stride = (long)p->num_q_heads * p->head_dim;
+    a.k_stride = a.v_stride = (long)p->num_kv_heads * p->head_dim;
+    a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.num_new = total; a.batch = p->batch; a.page_size = p->page_size; a.max_pages = p->max_pages_per_seq;
+    a.log2_theta = log2(p->rope_theta);
+    BatchLens bl;
+    fill_lens(&bl, p, h_cache_lens, h_new_offsets);
+    rope_append_kernel<__nv_bfloat16, true, BatchLens><<<total, 256, 0, (cudaStream_t)stream>>>(a, bl);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+evlnStatus_t evlnPagedStepAttention(evlnHandle_t h, const evlnPagedParams* p, const void* q_rot,
+                                    const void* k_pool, const void* v_pool, const int* h_cache_lens,
+                                    const int* h_new_offsets, const int* d_page_table, void* workspace,
+                                    size_t workspace_bytes, void* stream)
+{
+    evlnStatus_t s = check_paged_params(h, p, h_cache_lens, h_new_offsets);
+    if (s != EVLN_OK) return s;
+    const int total = h_new_offsets[p->batch];
+    if (total == 0) return EVLN_OK;
+    if (!q_rot || !k_pool || !v_pool || !d_page_table || !workspace) return EVLN_INVALID_VALUE;
+    if (!aligned16(q_rot) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(workspace))
+        return EVLN_INVALID_VALUE;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const long rows = (long)total * G;
+    int chunk, smax;
+    long items;
+    paged_schedule(h, p, h_cache_lens, h_new_offsets, &chunk, &smax, &items);
+    if (workspace_bytes < partial_bytes(smax, p->num_kv_heads, rows, 128)) return EVLN_WORKSPACE_TOO_SMALL;
+    if (items <= 0 || items > 0x7fffffffL) return EVLN_NOT_SUPPORTED;
+
+    CUtensorMap tm_q, tm_k, tm_v;
+    {
+        cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)p->num_kv_heads};
+        cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
+        cuuint32_t box[3] = {64, 128, 1};
+        if (!encode_map(h, &tm_q, q_rot, 3, dims, strides, box)) return EVLN_INVALID_VALUE;
+    }
+    {
+        cuuint64_t dims[4] = {128, 64, (cuuint64_t)p->num_kv_heads, (cuuint64_t)p->num_pages};
+        cuuint64_t strides[3] = {256, 64 * 256, (cuuint64_t)p->num_kv_heads * 64 * 256};
+        cuuint32_t box[4] = {64, 64, 1, 1};
+        if (!encode_map(h, &tm_k, k_pool, 4, dims, strides, box)) return EVLN_INVALID_VALUE;
+        if (!encode_map(h, &tm_v, v_pool, 4, dims, strides, box)) return EVLN_INVALID_VALUE;
+    }
+    const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(128.f);
+    TcAttnArgs a = {};
+    a.o_part = (float*)workspace;
+    a.lse_part = a.o_part + (size_t)smax * p->num_kv_heads * rows * 128;
+    a.page_table = d_page_table; a.status = h->d_status;
+    a.Hkv = p->num_kv_heads; a.G = G; a.rows = (int)rows;
+    a.batch = p->batch; a.max_pages = p->max_pages_per_seq; a.chunk_tiles = chunk;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    BatchLens bl;
+    fill_lens(&bl, p, h_cache_lens, h_new_offsets);
+    attn_tc_kernel<true, BatchLens><<<(int)items, kTcThreads, kTcSmemBytes, (cudaStream_t)stream>>>(
+        tm_q, tm_k, tm_v, a, bl);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+evlnStatus_t evlnPagedStepCombine(evlnHandle_t h, const evlnPagedParams* p, const void* workspace,
+                                  const int* h_cache_lens, const int* h_new_offsets, void* out, float* lse_out,
+                                  void* stream)
+{
+    evlnStatus_t s = check_paged_params(h, p, h_cache_lens, h_new_offsets);
+    if (s != EVLN_OK) return s;
+    const int total = h_new_offsets[p->batch];
+    if (total == 0) return EVLN_OK;
+    if (!workspace || !out || !aligned16(workspace) || !aligned16(out)) return EVLN_INVALID_VALUE;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const long rows = (long)total * G;
+    int chunk, smax;
+    long items;
+    paged_schedule(h, p, h_cache_lens, h_new_offsets, &chunk, &smax, &items);
+    CombineArgs a = {};
+    a.o_part = (const float*)workspace;
+    a.lse_part = a.o_part + (size_t)smax * p->num_kv_heads * rows * 128;
+    a.out = out; a.lse_out = lse_out;
+    a.Hkv = p->num_kv_heads; a.G = G; a.D = 128; a.rows = (int)rows; a.num_splits = smax;
+    a.batch = p->batch; a.unit_rows = kUnitRows; a.chunk_tiles = chunk;
+    BatchLens bl;
+    fill_lens(&bl, p, h_cache_lens, h_new_offsets);
+    return launch_combine<__nv_bfloat16>(h, a, 128, true, &bl, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,159 @@
+// Fused RoPE-rotate-and-append kernel (Sec. 3.2: contiguous position ids, rotation,
+// concatenation of the new frame with the reused cache).
+//
+// One CTA per new token.  Phase 1: D/2 threads form the token's angles phi_j = pos * theta^(-2j/D)
+// in double precision (pos reaches tens of thousands; a float angle would be off by ~1e-3 rad)
+// and leave cos/sin in shared memory for all heads.  Phase 2: every thread moves 16-byte
+// vectors: rotated query halves to the kv-head-grouped q_rot scratch, rotated key halves and
+// the unchanged values to the token's cache slot.  HBM-bound: each element is read once and
+// written once with 128-bit accesses.
+#pragma once
+
+#include "common.cuh"
+
+namespace evln {
+
+struct RopeArgs {
+    const void* q_new;
+    const void* k_new;
+    const void* v_new;
+    void* q_rot;
+    void* k_cache;      // contiguous: [Hkv, cap, D]; paged: pool [pages, Hkv, page, D]
+    void* v_cache;
+    const int* page_table;   // paged only: [batch, max_pages]
+    long q_stride, k_stride, v_stride;   // token strides in elements
+    int Hq, Hkv, D;
+    int cache_len;      // contiguous only
+    int num_new;        // contiguous: n; paged: total new tokens
+    int cache_cap;      // contiguous only
+    int batch, page_size, max_pages;     // paged only
+    double log2_theta;
+};
+
+// LensT is BatchLens for the paged kernel and NoLens (a stub) for the contiguous one.
+
+template <typename T, bool PAGED, typename LensT>
+__global__ void __launch_bounds__(256)
+rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
+{
+    constexpr int V = VecTraits<T>::kVec;
+    __shared__ double s_cos[128];
+    __shared__ double s_sin[128];
+
+    const int tok = blockIdx.x;           // index into the packed new tokens
+    const int D = a.D, half = D / 2;
+    const int G = a.Hq / a.Hkv;
+
+    int b = 0, i = tok, L = a.cache_len, n_b = a.num_new;
+    if (PAGED) {
+        int lo = 0, hi = a.batch;         // largest b with new_off[b] <= tok
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (lens.new_off[mid] <= tok) lo = mid; else hi = mid;
+        }
+        b = lo;
+        i = tok - lens.new_off[b];
+        L = lens.cache_len[b];
+        n_b = lens.new_off[b + 1] - lens.new_off[b];
+    }
+    const long pos = (long)L + i;
+
+    if (threadIdx.x < half) {
+        const int j = threadIdx.x;
+        double omega = exp2(-(2.0 * (double)j / (double)D) * a.log2_theta);
+        double s, c;
+        sincos((double)pos * omega, &s, &c);
+        s_cos[j] = c;
+        s_sin[j] = s;
+    }
+    __syncthreads();
+
+    // destination of this token's K/V row for kv head g (element offset)
+    long page_base = 0;     // paged: (page_id * Hkv) * page_size * D, slot within page
+    int slot = 0;
+    if (PAGED) {
+        int pg = a.page_table[(long)b * a.max_pages + (int)(pos / a.page_size)];
+        slot = (int)(pos % a.page_size);
+        page_base = (long)pg * a.Hkv * a.page_size * D;
+    }
+    auto kv_row = [&](int g) -> long {
+        if (PAGED) return page_base + ((long)g * a.page_size + slot) * D;
+        return ((long)g * a.cache_cap + pos) * D;
+    };
+
+    const T* q_tok = (const T*)a.q_new + (long)tok * a.q_stride;
+    const T* k_tok = (const T*)a.k_new + (long)tok * a.k_stride;
+    const T* v_tok = (const T*)a.v_new + (long)tok * a.v_stride;
+
+    const int vec_per_half = half / V;
+    const int q_items = a.Hq * vec_per_half;
+    const int k_items = a.Hkv * vec_per_half;
+    const int v_items = a.Hkv * (D / V);
+    const int items = q_items + k_items + v_items;
+    const long rows_per_head = PAGED ? (long)lens.new_off[a.batch] * G : (long)a.num_new * G;
+
+    for (int it = threadIdx.x; it < items; it += blockDim.x) {
+        if (it < q_items + k_items) {
+            const bool is_q = it < q_items;
+            const int e = is_q ? it : it - q_items;
+            const int h = e / vec_per_half;
+            const int j0 = (e % vec_per_half) * V;
+            const T* src = (is_q ? q_tok : k_tok) + (long)h * D;
+            T* dst;
+            if (is_q) {
+                const int g = h / G;
+                dst = (T*)a.q_rot + ((long)g * rows_per_head + (long)tok * G + (h % G)) * D;
+            } else {
+                dst = (T*)a.k_cache + kv_row(h);
+            }
+            uint4 lo_raw = *reinterpret_cast<const uint4*>(src + j0);
+            uint4 hi_raw = *reinterpret_cast<const uint4*>(src + j0 + half);
+            const T* lo = reinterpret_cast<const T*>(&lo_raw);
+            const T* hi = reinterpret_cast<const T*>(&hi_raw);
+            uint4 out_lo_raw, out_hi_raw;
+            T* out_lo = reinterpret_cast<T*>(&out_lo_raw);
+            T* out_hi = reinterpret_cast<T*>(&out_hi_raw);
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                if (sizeof(T) == 4) {
+                    // fp32 storage: products in double, one rounding to float
+                    double c = s_cos[j0 + v], s = s_sin[j0 + v];
+                    double x0 = (double)to_float(lo[v]), x1 = (double)to_float(hi[v]);
+                    from_float((float)(x0 * c - x1 * s), out_lo[v]);
+                    from_float((float)(x1 * c + x0 * s), out_hi[v]);
+                } else {
+                    float c = (float)s_cos[j0 + v], s = (float)s_sin[j0 + v];
+                    float x0 = to_float(lo[v]), x1 = to_float(hi[v]);
+                    from_float(fmaf(x0, c, -x1 * s), out_lo[v]);
+                    from_float(fmaf(x1, c, x0 * s), out_hi[v]);
+                }
+            }
+            *reinterpret_cast<uint4*>(dst + j0) = out_lo_raw;
+            *reinterpret_cast<uint4*>(dst + j0 + half) = out_hi_raw;
+        } else {
+            const int e = it - q_items - k_items;
+            const int g = e / (D / V);
+            const int d0 = (e % (D / V)) * V;
+            uint4 raw = *reinterpret_cast<const uint4*>(v_tok + (long)g * D + d0);
+            *reinterpret_cast<uint4*>((T*)a.v_cache + kv_row(g) + d0) = raw;
+        }
+    }
+
+    if (PAGED && i == n_b - 1 && slot + 1 < a.page_size) {
+        // the episode's last page is only partly filled: clear the value slots behind the last
+        // token so that a tile load of the whole page never brings in stale bits
+        const int tail = a.page_size - (slot + 1);
+        const int vec_per_row = D / V;
+        const int total = a.Hkv * tail * vec_per_row;
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        for (int it = threadIdx.x; it < total; it += blockDim.x) {
+            const int g = it / (tail * vec_per_row);
+            const int r = it % (tail * vec_per_row);
+            const int s2 = slot + 1 + r / vec_per_row;
+            const int d0 = (r % vec_per_row) * V;
+            *reinterpret_cast<uint4*>((T*)a.v_cache + page_base + ((long)g * a.page_size + s2) * D + d0) = zero;
+        }
+    }
+}
+
+}  // namespace evln

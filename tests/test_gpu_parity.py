@@ -1,0 +1,209 @@
+"""GPU parity: the CUDA path, called through the C-ABI, against the fp64 CPU oracle on the
+same seeded inputs.  Tolerances: appended K within 1 bf16 ulp (1e-6 abs for fp32), V
+bit-exact, attention output max-abs 1e-2 and mean-abs 1e-3 for bf16 (1e-5 for fp32), plus a
+relative Frobenius gate of 1e-2 because the absolute gates are loose at the small input
+scale of the 7B / 70B workloads."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import step_oracle as so
+from paper_2512_10310_b200 import binding as B
+from paper_2512_10310_b200 import workloads as W
+from tests.helpers import GpuStep, check_cache, check_output, f64, oracle_step
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def handle():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    h = B.evlnCreate(0)
+    yield h
+    B.evlnDestroy(h)
+
+
+def _run(handle, cfg, kernel=B.EVLN_KERNEL_AUTO, num_splits=0, extra_cap=37, lse_tol=1e-3, rel_tol=1e-2,
+         inputs=None, round_q=False, abs_tol=1e-2):
+    x = inputs or W.make_step_inputs(cfg)
+    L, n = cfg.cache_len, cfg.num_new
+    gs = GpuStep(handle, cfg.dtype, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n + extra_cap,
+                 cfg.rope_theta, n, num_splits=num_splits, kernel=kernel)
+    gs.load_cache(x["k_cache"], x["v_cache"])
+    g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
+    r = oracle_step(cfg.dtype, x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L,
+                    cfg.rope_theta)
+    check_cache(gs, r, L, n)
+    ref_out, ref_lse = r["out"], r["lse"]
+    if round_q:
+        # the tensor-core operand is the bf16-rounded rotated query: feed the oracle the same
+        # rounded q so that the comparison isolates the kernel from that input rounding
+        ref_out, ref_lse = so.attend_range(so.round_bf16(r["q_rot"]), r["k_cache"], r["v_cache"], L, 0, L + n)
+    check_output(cfg.dtype, g["out"], g["lse"], ref_out, ref_lse, lse_tol=lse_tol, rel_tol=rel_tol,
+                 abs_tol=abs_tol)
+    # rotated queries: bf16 rounding of the oracle's q_rot, at most one ulp apart
+    if cfg.dtype == "bf16":
+        from tests.helpers import bf16_ulp_distance
+        assert bf16_ulp_distance(g["q_rot"], so.round_bf16(r["q_rot"])).max() <= 1
+    else:
+        assert np.abs(f64(g["q_rot"]) - r["q_rot"]).max() <= 1e-6
+    return g, r
+
+
+def test_tiny_fp32_step(handle):
+    _run(handle, W.TINY_F32)
+
+
+@pytest.mark.parametrize("splits", [1, 3])
+def test_tiny_fp32_step_forced_splits(handle, splits):
+    _run(handle, W.TINY_F32, num_splits=splits)
+
+
+def test_simt_kernel_bf16_small(handle):
+    cfg = dataclasses.replace(W.STEP_7B, name="simt_small", cache_len=300, num_new=50)
+    _run(handle, cfg, kernel=B.EVLN_KERNEL_SIMT)
+
+
+def test_simt_kernel_bf16_d64(handle):
+    cfg = W.StepConfig("d64", "bf16", 4, 2, 64, 200, 33, 1e4, 0.3, 11)
+    _run(handle, cfg)
+
+
+# ---- tensor-core kernel ---------------------------------------------------------------------
+
+@pytest.mark.parametrize("L,n,splits", [
+    (0, 128, 1),          # instruction prefill, one exact tile pair per head... (G=7 -> ragged rows)
+    (0, 5, 0),            # shorter than one KV tile
+    (100, 1, 1),          # a single new token
+    (128, 37, 2),         # second query tile absent (259 rows -> 1.02 units)
+    (300, 50, 0),
+    (1000, 196, 3),
+    (2047, 130, 5),       # cache length not a multiple of anything
+])
+def test_tc_kernel_shapes(handle, L, n, splits):
+    cfg = dataclasses.replace(W.STEP_7B, name=f"tc_{L}_{n}", cache_len=L, num_new=n, seed=100 + L + n)
+    _run(handle, cfg, num_splits=splits)
+
+
+def test_tc_kernel_more_splits_than_tiles(handle):
+    cfg = dataclasses.replace(W.STEP_7B, name="oversplit", cache_len=200, num_new=20, seed=5)
+    _run(handle, cfg, num_splits=7)       # 2 KV tiles, 7 splits: five splits are empty
+
+
+def test_tc_kernel_sharp_logits(handle):
+    # unit-variance q and k: logits ~ N(0,1), softmax far from uniform
+    cfg = dataclasses.replace(W.STEP_7B, name="sharp", cache_len=1500, num_new=100, input_scale=1.0, seed=6)
+    _run(handle, cfg, lse_tol=2e-2, rel_tol=1.5e-2)
+
+
+def test_tc_kernel_planted_high_logit_keys(handle):
+    # a few cached keys aligned with the queries dominate the softmax; the running maximum has to
+    # move by far more than the lazy-rescale threshold in a late tile
+    cfg = dataclasses.replace(W.STEP_7B, name="planted", cache_len=900, num_new=64, input_scale=1.0, seed=7)
+    x = W.make_step_inputs(cfg)
+    x["k_cache"][850:853] *= 6.0
+    x["k_new"][40:42] *= 8.0
+    # logits reach ~30 here, so the bf16 rounding of the rotated query alone moves them by ~1e-2;
+    # outputs are O(1): the absolute gate scales with them
+    _run(handle, cfg, num_splits=1, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2)
+    _run(handle, cfg, num_splits=3, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2)
+
+
+def test_tc_matches_simt_kernel_on_device(handle):
+    cfg = dataclasses.replace(W.STEP_7B, name="cross", cache_len=700, num_new=90, seed=8)
+    a, _ = _run(handle, cfg)
+    b, _ = _run(handle, cfg, kernel=B.EVLN_KERNEL_SIMT)
+    assert (a["out"].float() - b["out"].float()).abs().max().item() <= 2e-3
+
+
+def test_step_7b_full(handle):
+    g, _ = _run(handle, W.STEP_7B)
+    assert g["splits"] >= 2
+
+
+def test_results_are_bitwise_reproducible(handle):
+    cfg = dataclasses.replace(W.STEP_7B, name="repro", cache_len=1024, num_new=196, seed=9)
+    a, _ = _run(handle, cfg)
+    b, _ = _run(handle, cfg)
+    assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
+    assert torch.equal(a["lse"], b["lse"])
+
+
+def test_chained_steps_reuse_the_cache(handle):
+    # instruction prefill then three frames through the same cache: equals the oracle chain
+    cfg = dataclasses.replace(W.STEP_7B, name="chain", cache_len=0, num_new=0, seed=10)
+    chunks = [256, 204, 204, 204]
+    T = sum(chunks)
+    gs = GpuStep(handle, "bf16", 28, 4, 128, T + 5, cfg.rope_theta, max(chunks))
+    kc = np.zeros((T + 5, 4, 128))
+    vc = np.zeros((T + 5, 4, 128))
+    L = 0
+    for s, n in enumerate(chunks):
+        x = W.make_new_tokens(dataclasses.replace(cfg, num_new=n, seed=1000 + s))
+        g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
+        r = so.step(f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"]), kc, vc, L, cfg.rope_theta,
+                    storage="bf16")
+        check_output("bf16", g["out"], g["lse"], r["out"], r["lse"])
+        L += n
+    from tests.helpers import bf16_ulp_distance
+    assert bf16_ulp_distance(gs.k_cache[:, :T].permute(1, 0, 2), kc[:T]).max() <= 1
+    assert np.array_equal(f64(gs.v_cache[:, :T].permute(1, 0, 2)), vc[:T])
+
+
+def test_long_70b_sampled_rows(handle):
+    # full-size launch; the oracle computes a sample of query tokens one by one
+    cfg = W.LONG_70B
+    x = W.make_step_inputs(cfg)
+    L, n = cfg.cache_len, cfg.num_new
+    gs = GpuStep(handle, "bf16", cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n, cfg.rope_theta, n)
+    gs.load_cache(x["k_cache"], x["v_cache"])
+    g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
+    kc = np.zeros((L + n, cfg.num_kv_heads, cfg.head_dim))
+    vc = np.zeros_like(kc)
+    kc[:L], vc[:L] = f64(x["k_cache"]), f64(x["v_cache"])
+    kc[L:] = so.round_bf16(so.rope(f64(x["k_new"]), L, cfg.rope_theta))
+    vc[L:] = f64(x["v_new"])
+    q_rot = so.rope(f64(x["q_new"]), L, cfg.rope_theta)
+    from tests.helpers import bf16_ulp_distance
+    assert bf16_ulp_distance(gs.k_cache[:, L:].permute(1, 0, 2), kc[L:]).max() <= 1
+    assert np.array_equal(f64(gs.v_cache[:, L:].permute(1, 0, 2)), vc[L:])
+    for i in (0, 1, 127, 128, 200, 255):
+        o, l = so.attend_range(q_rot[i:i + 1], kc, vc, L + i, 0, L + i + 1)
+        check_output("bf16", g["out"][i:i + 1], g["lse"][i:i + 1], o, l)
+
+
+# ---- boundary behaviour (argument errors launch nothing) ------------------------------------
+
+def test_argument_errors(handle):
+    p = B.step_params("bf16", 28, 4, 128, 10, 5, 12, 1e6)
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnStepWorkspaceSize(handle, p)
+    assert e.value.status == B.EVLN_CACHE_FULL
+    p = B.step_params("bf16", 28, 5, 128, 10, 5, 100, 1e6)
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnStepWorkspaceSize(handle, p)
+    assert e.value.status == B.EVLN_INVALID_VALUE
+    p = B.step_params("bf16", 28, 4, 96, 10, 5, 100, 1e6)
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnStepWorkspaceSize(handle, p)
+    assert e.value.status == B.EVLN_NOT_SUPPORTED
+    # misaligned pointer, null pointer, short workspace
+    p = B.step_params("bf16", 28, 4, 128, 10, 5, 100, 1e6)
+    buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda:0")
+    base = buf.data_ptr()
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnRopeAppend(handle, p, base + 2, base, base, base, base, base, strides=(28 * 128, 512, 512))
+    assert e.value.status == B.EVLN_INVALID_VALUE
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnRopeAppend(handle, p, None, base, base, base, base, base, strides=(28 * 128, 512, 512))
+    assert e.value.status == B.EVLN_INVALID_VALUE
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnStepAttention(handle, p, base, base, base, base, workspace_bytes=64)
+    assert e.value.status == B.EVLN_WORKSPACE_TOO_SMALL
+    # n = 0 is a no-op
+    p0 = B.step_params("bf16", 28, 4, 128, 10, 0, 100, 1e6)
+    B.evlnRopeAppend(handle, p0, base, base, base, base, base, base, strides=(28 * 128, 512, 512))
+    assert B.evlnGetDeviceStatus(handle) == 0
