@@ -125,8 +125,8 @@ evlnStatus_t evlnStepQRotSize(evlnHandle_t handle, const evlnStepParams* params,
 /* Step 1 (Sec. 3.2: contiguous position ids, RoPE, concatenation with the cache).
  * Rotates the new queries at positions L+i into q_rot (grouped by kv head), rotates the new
  * keys and stores them, with the values copied bit-exactly, into cache slots L .. L+n-1.
- * Angles are formed in double precision, products in float (double for EVLN_F32), one
- * rounding to the storage dtype.  Slots outside L .. L+n-1 are not touched.
+ * Angles, sines/cosines and the rotation products are formed in double precision and then
+ * rounded to the storage dtype.  Slots outside L .. L+n-1 are not touched.
  * Errors: EVLN_CACHE_FULL if L+n > cache_capacity; n = 0 returns EVLN_OK and launches nothing. */
 evlnStatus_t evlnRopeAppend(evlnHandle_t handle, const evlnStepParams* params,
                             const void* q_new, const void* k_new, const void* v_new,

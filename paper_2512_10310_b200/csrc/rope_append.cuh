@@ -3,7 +3,7 @@
 //
 // One CTA per new token.  Phase 1: D/2 threads form the token's angles phi_j = pos * theta^(-2j/D)
 // in double precision (pos reaches tens of thousands; a float angle would be off by ~1e-3 rad)
-// and leave cos/sin in shared memory for all heads.  Phase 2: every thread moves 16-byte
+// and leave cos/sin (double) in shared memory for all heads.  Phase 2: every thread moves 16-byte
 // vectors: rotated query halves to the kv-head-grouped q_rot scratch, rotated key halves and
 // the unchanged values to the token's cache slot.  HBM-bound: each element is read once and
 // written once with 128-bit accesses.
@@ -115,18 +115,12 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
             T* out_hi = reinterpret_cast<T*>(&out_hi_raw);
 #pragma unroll
             for (int v = 0; v < V; ++v) {
-                if (sizeof(T) == 4) {
-                    // fp32 storage: products in double, one rounding to float
-                    double c = s_cos[j0 + v], s = s_sin[j0 + v];
-                    double x0 = (double)to_float(lo[v]), x1 = (double)to_float(hi[v]);
-                    from_float((float)(x0 * c - x1 * s), out_lo[v]);
-                    from_float((float)(x1 * c + x0 * s), out_hi[v]);
-                } else {
-                    float c = (float)s_cos[j0 + v], s = (float)s_sin[j0 + v];
-                    float x0 = to_float(lo[v]), x1 = to_float(hi[v]);
-                    from_float(fmaf(x0, c, -x1 * s), out_lo[v]);
-                    from_float(fmaf(x1, c, x0 * s), out_hi[v]);
-                }
+                // products and the difference in double (a float product loses bits exactly where
+                // x0*c and x1*s cancel), then one rounding to float and one to the storage dtype
+                const double c = s_cos[j0 + v], s = s_sin[j0 + v];
+                const double x0 = (double)to_float(lo[v]), x1 = (double)to_float(hi[v]);
+                from_float((float)(x0 * c - x1 * s), out_lo[v]);
+                from_float((float)(x1 * c + x0 * s), out_hi[v]);
             }
             *reinterpret_cast<uint4*>(dst + j0) = out_lo_raw;
             *reinterpret_cast<uint4*>(dst + j0 + half) = out_hi_raw;
