@@ -30,6 +30,7 @@ import numpy as np
 import torch
 
 from paper_2512_10310_b200 import workloads as W
+from paper_2512_10310_b200.replicas import aggregate_steps_per_s, max_over_ranks as _max_over_ranks
 
 RING_LAYERS = 32            # independent layer caches cycled through (footprint > L2)
 L2_BYTES = 126 * 2 ** 20
@@ -204,11 +205,7 @@ def run_ours(args, rank, world, local_rank, dist):
             dist.barrier()
 
     def max_over_ranks(x):
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return _max_over_ranks(x, dist, dev)
 
     steps = max(RING_LAYERS, (args.steps // RING_LAYERS) * RING_LAYERS)
     warm = max(3 * RING_LAYERS, -(-args.warmup // RING_LAYERS) * RING_LAYERS)
@@ -268,7 +265,7 @@ def run_ours(args, rank, world, local_rank, dist):
         },
         "tflops": round(flops / (us_step * 1e-6) / 1e12 * world, 2),
         "gbs": round(abytes / (us_step * 1e-6) / 1e9 * world, 1),
-        "steps_per_s": round(world / (us_step * 1e-6), 1),
+        "steps_per_s": round(aggregate_steps_per_s(us_step, world), 1),
         "step_roofline_frac": round(max(t_flop_us, t_hbm_us) / us_step, 4),
         "roofline": {
             "kernel": "attn_tc_kernel (evlnStepAttention)", "bound": "tensor",
@@ -324,9 +321,11 @@ def cpu_baseline_full_step(cfg):
     vc = np.zeros_like(kc)
     kc[:L], vc[:L] = f64(x["k_cache"]), f64(x["v_cache"])
     q, k, v = f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"])
+    reps = 5
     t0 = time.perf_counter()
-    so.step(q, k, v, kc, vc, L, cfg.rope_theta, storage="bf16")
-    dt = time.perf_counter() - t0
+    for _ in range(reps):
+        so.step(q, k, v, kc, vc, L, cfg.rope_theta, storage="bf16")
+    dt = (time.perf_counter() - t0) / reps
     return dt, so.num_threads()
 
 
@@ -394,7 +393,7 @@ def main():
             dt, threads = cpu_baseline_full_step(W.STEP_7B)
             line["cpu_baseline"] = {
                 "value": round(dt * 1e6, 1), "unit": "us/step", "cores": threads, "kind": "oracle",
-                "sample": "1 full step of the same workload (all 196 tokens x 28 heads), rotate + append + attention",
+                "sample": "mean of 5 full steps of the same workload (all 196 tokens x 28 heads), rotate + append + attention",
             }
         print(json.dumps(line), flush=True)
     if dist is not None:

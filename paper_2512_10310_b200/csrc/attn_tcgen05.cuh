@@ -31,6 +31,12 @@
 
 namespace evln {
 
+#ifdef EVLN_TIMELINE
+#define EVLN_STAMP(slot) do { if (a.timeline && (slot) < 32) a.timeline[(long)blockIdx.x * 32 + (slot)] = clock64(); } while (0)
+#else
+#define EVLN_STAMP(slot) do { } while (0)
+#endif
+
 constexpr int kTcThreads = 384;
 constexpr int kStages = 5;
 constexpr int kTileBytes = kTileN * 128 * 2;          // 128 rows x 128 channels x bf16
@@ -56,6 +62,9 @@ struct TcAttnArgs {
     int units_per_head;       // contiguous only
     int batch, max_pages, chunk_tiles;   // paged only
     float scale_log2;         // softmax scale * log2(e)
+#ifdef EVLN_TIMELINE
+    long long* timeline;      // debug builds only: 32 clock stamps per CTA
+#endif
 };
 
 // --- descriptors --------------------------------------------------------------------------
@@ -187,6 +196,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + kSmemBarOff + (tmem_slot - bar_base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) EVLN_STAMP(0);
 
     const WorkItem w = decode_work<PAGED, LensT>(a, lens, blockIdx.x);
     if (PAGED && w.b < 0) return;
@@ -239,6 +249,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __syncthreads();
     ptx::fence_after_sync();
     const uint32_t tmem = *s_tmem;
+    if (threadIdx.x == 0) EVLN_STAMP(1);
 
     if (warp == 0) {
         // ================= TMA producer =================
@@ -396,6 +407,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             ptx::fence_after_sync();
+            if (warp == 4 && lane == 0) EVLN_STAMP(2 + 2 * it);
 
             const int j = w.j0 + it;
             const int lim = bound - j * kTileN;            // columns 0..lim are visible
@@ -463,6 +475,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ptx::tmem_st_wait();
             ptx::fence_before_sync();
             ptx::mbar_arrive(bar_p_full + 8 * x);
+            if (warp == 4 && lane == 0) EVLN_STAMP(3 + 2 * it);
         }
 
         if (ok) {
@@ -471,6 +484,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         if (ok) {
             ptx::fence_after_sync();
+            if (warp == 4 && lane == 0) EVLN_STAMP(28);
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             const long prow = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + r_local;
             float4* dst = reinterpret_cast<float4*>(a.o_part + prow * 128);
@@ -489,6 +503,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             if (row_valid)
                 a.lse_part[prow] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            if (warp == 4 && lane == 0) EVLN_STAMP(29);
         }
     }
 
@@ -498,6 +513,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (warp == 1) {
         ptx::fence_after_sync();
         ptx::tmem_dealloc(tmem, 512);
+        if (lane == 0) EVLN_STAMP(30);
     }
 }
 

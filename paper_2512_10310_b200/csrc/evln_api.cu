@@ -31,6 +31,11 @@ struct evlnContext {
     EncodeTiledFn encode;
 };
 
+#ifdef EVLN_TIMELINE
+static long long* g_timeline = nullptr;
+extern "C" void evlnDebugSetTimeline(void* p) { g_timeline = (long long*)p; }
+#endif
+
 namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -382,6 +387,9 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
         a.cache_len = p->cache_len; a.num_new = p->num_new; a.num_splits = S;
         a.units_per_head = ceil_div(R, kUnitRows);
         a.scale_log2 = scale * 1.4426950408889634f;
+#ifdef EVLN_TIMELINE
+        a.timeline = g_timeline;
+#endif
         NoLens nl = {};
         const int grid = S * p->num_kv_heads * a.units_per_head;
         attn_tc_kernel<false, NoLens><<<grid, kTcThreads, kTcSmemBytes, st>>>(tm_q, tm_k, tm_v, a, nl);
