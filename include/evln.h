@@ -172,6 +172,42 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t handle, const evlnPagedParams* pa
                                   const int* h_new_offsets, void* out, float* lse_out,
                                   void* stream);
 
+/* ---- allocation-free variant ------------------------------------------------------------ */
+
+/* Largest split workspace the allocation-free call can serve (bytes of its built-in scratch). */
+#define EVLN_NOALLOC_SCRATCH_BYTES (32u << 20)
+
+/* Attention + combine of one step for callers that cannot allocate device memory.  (The paper
+ * has no counterpart for this call; it exists for deployment.)
+ *
+ * Who needs it: a host process that has handed all device memory to its own arena at start-up
+ * (an inference server, a robot's control process with a fixed memory budget), or code that
+ * runs where cudaMalloc is unwelcome because it synchronises the whole device and may fail
+ * late.  Such a caller can neither create a handle (evlnCreate allocates its status word) nor
+ * size and allocate the split workspace.  This call needs neither: it takes no handle, and the
+ * per-split partial results go to a scratch array that is part of the library image itself
+ * (EVLN_NOALLOC_SCRATCH_BYTES of device memory, held by every GPU that loads the library until
+ * the process exits).  The caller passes only inputs and outputs:
+ *   q_rot, k_cache, v_cache: the rotated queries and the cache exactly as evlnRopeAppend leaves
+ *   them (that call allocates nothing either, but wants a handle made while allocating was
+ *   still allowed, e.g. at start-up; the workspace size, in contrast, changes with L);
+ *   out [n, Hq, D], lse_out [n, Hq] or NULL: as for evlnStepCombine.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *
+ * Set-up: the first call on each device (with that device current) looks up the scratch
+ * array's device address and the device's properties once; make that first call outside any
+ * stream capture.  Later calls on that device only validate and launch.
+ * Limits and errors: parameters whose split workspace (evlnStepWorkspaceSize) exceeds
+ * EVLN_NOALLOC_SCRATCH_BYTES are rejected with EVLN_WORKSPACE_TOO_SMALL and nothing is
+ * launched; other errors as for evlnStepAttention / evlnStepCombine.
+ * Sharing: every call on a device uses the same scratch array, which keeps the previous
+ * call's contents (each call overwrites every partial it later reads, so nothing needs
+ * clearing).  Two such calls that overlap on the GPU (different streams, or different host
+ * threads) race on it: serialise them.                                                        */
+evlnStatus_t evlnStepAttentionNoAlloc(const evlnStepParams* params, const void* q_rot,
+                                      const void* k_cache, const void* v_cache, void* out,
+                                      float* lse_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

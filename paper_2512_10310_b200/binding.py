@@ -28,7 +28,9 @@ EXPORTS = [
     "evlnStepNumSplits", "evlnStepWorkspaceSize", "evlnStepQRotSize",
     "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine",
     "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
+    "evlnStepAttentionNoAlloc",
 ]
+EVLN_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
 class evlnStepParams(Structure):
@@ -103,6 +105,7 @@ def lib():
         L.evlnPagedStepAttention.argtypes = [c_void_p, gp, c_void_p, c_void_p, c_void_p, ip, ip, c_void_p,
                                              c_void_p, c_size_t, c_void_p]
         L.evlnPagedStepCombine.argtypes = [c_void_p, gp, c_void_p, ip, ip, c_void_p, c_void_p, c_void_p]
+        L.evlnStepAttentionNoAlloc.argtypes = [pp, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         for name in EXPORTS:
             if name != "evlnGetErrorString":
                 getattr(L, name).restype = c_int
@@ -253,3 +256,12 @@ def evlnPagedStepCombine(handle, params, workspace, cache_lens, new_offsets, out
     _check(lib().evlnPagedStepCombine(handle, byref(params), _ptr(workspace), _ints(cache_lens),
                                       _ints(new_offsets), _ptr(out), _ptr(lse_out), _stream(stream)),
            "evlnPagedStepCombine")
+
+
+def evlnStepAttentionNoAlloc(params, q_rot, k_cache, v_cache, out, lse_out=None, stream=None):
+    """Attention + combine without a handle or a caller workspace: the split partials go to a
+    scratch array built into the library (at most EVLN_NOALLOC_SCRATCH_BYTES).  For callers that
+    must not allocate device memory; calls sharing a device must not overlap."""
+    _check(lib().evlnStepAttentionNoAlloc(byref(params), _ptr(q_rot), _ptr(k_cache), _ptr(v_cache),
+                                          _ptr(out), _ptr(lse_out), _stream(stream)),
+           "evlnStepAttentionNoAlloc")

@@ -552,3 +552,77 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t h, const evlnPagedParams* p, cons
 }
 
 }  // extern "C"
+
+// ---- allocation-free variant --------------------------------------------------------------
+
+// Scratch for the split partials of evlnStepAttentionNoAlloc, part of the library image: every
+// device that loads the library holds these bytes until the process exits.  In host code the
+// names below are only stand-ins for the device objects; their device addresses come from
+// cudaGetSymbolAddress (once per device) and are what the kernels receive.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[EVLN_NOALLOC_SCRATCH_BYTES];
+static __device__ __align__(256) int g_noalloc_status[64];
+
+namespace {
+constexpr int kMaxDevices = 64;
+struct NoAllocDevice {
+    bool ready;
+    evlnContext ctx;          // plain struct used as the handle of the regular entry points
+    void* scratch;
+};
+NoAllocDevice g_noalloc_dev[kMaxDevices];
+
+// First call on a device: resolve device addresses and properties.  Allocates nothing.
+evlnStatus_t noalloc_setup(int device, NoAllocDevice** out)
+{
+    if (device < 0 || device >= kMaxDevices) return EVLN_NOT_SUPPORTED;
+    NoAllocDevice* d = &g_noalloc_dev[device];
+    if (!d->ready) {
+        cudaDeviceProp prop;
+        cudaError_t e = cudaGetDeviceProperties(&prop, device);
+        if (e != cudaSuccess) return EVLN_CUDA_ERROR;
+        if (prop.major != 10) return EVLN_NOT_SUPPORTED;
+        void* scratch = nullptr;
+        void* status = nullptr;
+        e = cudaGetSymbolAddress(&scratch, g_noalloc_scratch);
+        if (e != cudaSuccess || !scratch) return EVLN_CUDA_ERROR;
+        e = cudaGetSymbolAddress(&status, g_noalloc_status);
+        if (e != cudaSuccess || !status) return EVLN_CUDA_ERROR;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return EVLN_CUDA_ERROR;
+        e = cudaFuncSetAttribute(attn_tc_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kTcSmemBytes);
+        if (e != cudaSuccess) return EVLN_CUDA_ERROR;
+        d->ctx.device = device;
+        d->ctx.num_sms = prop.multiProcessorCount;
+        d->ctx.last_cuda_error = 0;
+        d->ctx.d_status = static_cast<int*>(status);
+        d->ctx.encode = reinterpret_cast<EncodeTiledFn>(fn);
+        d->scratch = scratch;
+        d->ready = true;
+    }
+    *out = d;
+    return EVLN_OK;
+}
+}  // namespace
+
+extern "C" evlnStatus_t evlnStepAttentionNoAlloc(const evlnStepParams* p, const void* q_rot, const void* k_cache,
+                                                 const void* v_cache, void* out, float* lse_out, void* stream)
+{
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return EVLN_CUDA_ERROR;
+    NoAllocDevice* d = nullptr;
+    evlnStatus_t s = noalloc_setup(device, &d);
+    if (s != EVLN_OK) return s;
+    evlnHandle_t h = &d->ctx;
+    size_t need = 0;
+    s = evlnStepWorkspaceSize(h, p, &need);
+    if (s != EVLN_OK) return s;
+    if (need > (size_t)EVLN_NOALLOC_SCRATCH_BYTES) return EVLN_WORKSPACE_TOO_SMALL;
+    if (p->num_new == 0) return EVLN_OK;
+    if (!out) return EVLN_INVALID_VALUE;
+    s = evlnStepAttention(h, p, q_rot, k_cache, v_cache, d->scratch, (size_t)EVLN_NOALLOC_SCRATCH_BYTES, stream);
+    if (s != EVLN_OK) return s;
+    return evlnStepCombine(h, p, d->scratch, out, lse_out, stream);
+}
