@@ -1,0 +1,141 @@
+"""GPU parity of the paged batch path (evlnPaged*) against the oracle's paged wrapper."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import step_oracle as so
+from paper_2512_10310_b200 import binding as B
+from paper_2512_10310_b200 import workloads as W
+from tests.helpers import bf16_ulp_distance, check_output, f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def handle():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    h = B.evlnCreate(0)
+    yield h
+    B.evlnDestroy(h)
+
+
+def _gpu_paged(handle, cfg, x, kv_chunk_tiles=0):
+    dev = "cuda:0"
+    Bn, P = len(x["cache_lens"]), cfg.page_size
+    Hq, Hkv, D = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
+    max_pages = max(len(t) for t in x["page_table"]) + 3
+    table = torch.full((Bn, max_pages), -1, dtype=torch.int32)
+    for b, t in enumerate(x["page_table"]):
+        table[b, :len(t)] = torch.tensor(t, dtype=torch.int32)
+    table = table.clamp(min=0).to(dev)
+    # pool layout [pages, Hkv, P, D]; every slot that holds no token starts as NaN so that any
+    # leak of an unwritten slot into the result is caught
+    k_pool = torch.full((x["num_pages"], Hkv, P, D), float("nan"), dtype=torch.bfloat16, device=dev)
+    v_pool = torch.full((x["num_pages"], Hkv, P, D), float("nan"), dtype=torch.bfloat16, device=dev)
+    for b, L in enumerate(x["cache_lens"]):
+        for pi in range((L + P - 1) // P):
+            pg = x["page_table"][b][pi]
+            cnt = min(P, L - pi * P)
+            k_pool[pg, :, :cnt] = x["k_pool"][pg, :cnt].to(dev).permute(1, 0, 2)
+            v_pool[pg, :, :cnt] = x["v_pool"][pg, :cnt].to(dev).permute(1, 0, 2)
+    p = B.paged_params(Hq, Hkv, D, Bn, P, x["num_pages"], max_pages, cfg.rope_theta, kv_chunk_tiles=kv_chunk_tiles)
+    lens, offs = x["cache_lens"], x["new_offsets"]
+    total = offs[-1]
+    q, k, v = (x[s].to(dev) for s in ("q_new", "k_new", "v_new"))
+    q_rot = torch.empty(total * Hq * D * 2 + 256, dtype=torch.uint8, device=dev)
+    ws = torch.empty(B.evlnPagedWorkspaceSize(handle, p, lens, offs), dtype=torch.uint8, device=dev)
+    out = torch.full((total, Hq, D), float("nan"), dtype=torch.bfloat16, device=dev)
+    lse = torch.full((total, Hq), float("nan"), dtype=torch.float32, device=dev)
+    B.evlnPagedRopeAppend(handle, p, q, k, v, lens, offs, table, q_rot, k_pool, v_pool)
+    B.evlnPagedStepAttention(handle, p, q_rot, k_pool, v_pool, lens, offs, table, ws)
+    B.evlnPagedStepCombine(handle, p, ws, lens, offs, out, lse)
+    assert B.evlnGetDeviceStatus(handle) == 0
+    return out, lse, k_pool, v_pool
+
+
+def _check_pools(x, cfg, k_pool, v_pool, ok_pool, ov_pool):
+    P = cfg.page_size
+    for b, L in enumerate(x["cache_lens"]):
+        n = x["new_offsets"][b + 1] - x["new_offsets"][b]
+        for t in list(range(L, L + n)):
+            pg, sl = x["page_table"][b][t // P], t % P
+            assert bf16_ulp_distance(k_pool[pg, :, sl], ok_pool[pg, sl]).max() <= 1
+            assert np.array_equal(f64(v_pool[pg, :, sl]), ov_pool[pg, sl])
+        # value slots behind the last token of the last page are cleared
+        last = L + n
+        if last % P:
+            pg = x["page_table"][b][last // P]
+            assert bool((v_pool[pg, :, last % P:] == 0).all())
+
+
+def test_paged_small_ragged_batch(handle):
+    cfg = dataclasses.replace(W.PAGED_B16, name="paged_small", batch=5, seed=31)
+    lens = [0, 63, 64, 333, 1000]
+    news = [70, 1, 129, 37, 196]
+    x = W.make_paged_inputs(cfg, lens=lens, num_new=news)
+    for chunk in (0, 2):
+        out, lse, k_pool, v_pool = _gpu_paged(handle, cfg, x, kv_chunk_tiles=chunk)
+        okp, ovp = f64(x["k_pool"]), f64(x["v_pool"])
+        ref_out, ref_lse = so.step_paged(f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"]), okp, ovp,
+                                         x["page_table"], lens, x["new_offsets"], cfg.rope_theta, storage="bf16")
+        check_output("bf16", out, lse, ref_out, ref_lse)
+        _check_pools(x, cfg, k_pool, v_pool, okp, ovp)
+
+
+def test_paged_equals_contiguous_on_device(handle):
+    # the same episode through the contiguous entry points gives the same bits up to split order
+    cfg = dataclasses.replace(W.PAGED_B16, name="paged_vs_contig", batch=1, seed=32)
+    x = W.make_paged_inputs(cfg, lens=[777], num_new=[150])
+    out, lse, _, _ = _gpu_paged(handle, cfg, x)
+    from tests.helpers import GpuStep
+    gs = GpuStep(handle, "bf16", cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, 777 + 150, cfg.rope_theta, 150)
+    P = cfg.page_size
+    kc = torch.cat([x["k_pool"][pg] for pg in x["page_table"][0]])[:777]
+    vc = torch.cat([x["v_pool"][pg] for pg in x["page_table"][0]])[:777]
+    gs.load_cache(kc, vc)
+    g = gs.step(777, x["q_new"], x["k_new"], x["v_new"])
+    assert (g["out"].float() - out.float()).abs().max().item() <= 2e-4
+    assert (g["lse"] - lse).abs().max().item() <= 1e-5
+
+
+def test_paged_b16_full_size_sampled(handle):
+    # the full serving batch; the oracle checks sampled tokens of sampled episodes one by one
+    cfg = W.PAGED_B16
+    x = W.make_paged_inputs(cfg)
+    out, lse, k_pool, v_pool = _gpu_paged(handle, cfg, x)
+    P, theta = cfg.page_size, cfg.rope_theta
+    lens, offs = x["cache_lens"], x["new_offsets"]
+    order = np.argsort(lens)
+    for b in (int(order[0]), int(order[len(order) // 2]), int(order[-1])):
+        L, lo, hi = lens[b], offs[b], offs[b + 1]
+        n = hi - lo
+        pages = x["page_table"][b]
+        kc = np.zeros((L + n, cfg.num_kv_heads, cfg.head_dim))
+        vc = np.zeros_like(kc)
+        kc[:L] = f64(torch.cat([x["k_pool"][pg] for pg in pages])[:L])
+        vc[:L] = f64(torch.cat([x["v_pool"][pg] for pg in pages])[:L])
+        kc[L:] = so.round_bf16(so.rope(f64(x["k_new"][lo:hi]), L, theta))
+        vc[L:] = f64(x["v_new"][lo:hi])
+        q_rot = so.rope(f64(x["q_new"][lo:hi]), L, theta)
+        for i in (0, 18, 100, n - 1):
+            o, l = so.attend_range(q_rot[i:i + 1], kc, vc, L + i, 0, L + i + 1)
+            check_output("bf16", out[lo + i:lo + i + 1], lse[lo + i:lo + i + 1], o, l)
+        # appended slots of this episode
+        for t in (L, L + n - 1):
+            pg, sl = pages[t // P], t % P
+            assert bf16_ulp_distance(k_pool[pg, :, sl], kc[t]).max() <= 1
+            assert np.array_equal(f64(v_pool[pg, :, sl]), vc[t])
+
+
+def test_paged_argument_errors(handle):
+    p = B.paged_params(28, 4, 128, 2, 64, 10, 2, 1e6)
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnPagedWorkspaceSize(handle, p, [100, 100], [0, 10, 60])   # second episode needs 3 pages
+    assert e.value.status == B.EVLN_CACHE_FULL
+    p = B.paged_params(28, 4, 128, 2, 32, 10, 8, 1e6)
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnPagedWorkspaceSize(handle, p, [100, 100], [0, 10, 20])
+    assert e.value.status == B.EVLN_NOT_SUPPORTED
