@@ -29,6 +29,8 @@ __global__ void __launch_bounds__(128)
 attn_simt_kernel(const SimtAttnArgs a)
 {
     constexpr int C = D / 32;                 // output channels per lane
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ float s_q[4][D];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -32,7 +32,7 @@
 namespace evln {
 
 #ifdef EVLN_TIMELINE
-#define EVLN_STAMP(slot) do { if (a.timeline && (slot) < 32) a.timeline[(long)blockIdx.x * 32 + (slot)] = clock64(); } while (0)
+#define EVLN_STAMP(slot) do { if (a.timeline && (slot) < 64) a.timeline[(long)blockIdx.x * 64 + (slot)] = clock64(); } while (0)
 #else
 #define EVLN_STAMP(slot) do { } while (0)
 #endif
@@ -109,6 +109,57 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, int 
         }
     }
     return true;
+}
+
+// One lane polls, the warp shares the outcome (fewer pollers on the barrier word).
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, int code, int* status,
+                                          volatile int* s_abort, int lane)
+{
+    int r = 1;
+    if (lane == 0) r = wait_bounded(bar, parity, code, status, s_abort) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, r, 0) != 0;
+}
+
+// --- softmax pieces on one 32-column register block of a score row ---------------------------
+
+__device__ __forceinline__ void mask32(uint32_t (&s)[32], int lim)
+{
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+        if (e > lim) s[e] = 0xff800000u;
+}
+
+__device__ __forceinline__ void rowmax32(const uint32_t (&s)[32], float& m0, float& m1, float& m2, float& m3)
+{
+#pragma unroll
+    for (int e = 0; e < 32; e += 8) {
+        m0 = ptx::max3(m0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+        m1 = ptx::max3(m1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+        m2 = ptx::max3(m2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+        m3 = ptx::max3(m3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
+    }
+}
+
+// p = 2^(s*scale + negm) for 32 columns, accumulated into two packed sums, written to TMEM as
+// 16 columns of packed bf16 pairs
+__device__ __forceinline__ void exp32_store(const uint32_t (&s)[32], uint32_t taddr, uint64_t scale2,
+                                            uint64_t negm2, uint64_t& sum2a, uint64_t& sum2b)
+{
+    uint32_t packed[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        const uint64_t xa = ptx::fma2(ptx::pack2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), scale2, negm2);
+        const uint64_t xb = ptx::fma2(ptx::pack2(__uint_as_float(s[e + 2]), __uint_as_float(s[e + 3])), scale2, negm2);
+        float x0, x1, x2, x3;
+        ptx::unpack2(xa, x0, x1);
+        ptx::unpack2(xb, x2, x3);
+        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1), p2 = ptx::ex2(x2), p3 = ptx::ex2(x3);
+        sum2a = ptx::add2(sum2a, ptx::pack2(p0, p1));
+        sum2b = ptx::add2(sum2b, ptx::pack2(p2, p3));
+        packed[e >> 1] = ptx::pack_bf16x2(p0, p1);
+        packed[(e >> 1) + 1] = ptx::pack_bf16x2(p2, p3);
+    }
+    ptx::tmem_st16(taddr, packed);
 }
 
 // --- work decoding ------------------------------------------------------------------------
@@ -209,6 +260,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     // A split with no KV tiles (more splits than tiles): its partials are "empty".
     if (ntiles <= 0) {
+        ptx::grid_dependency_wait();
         if (warp >= 4 && warp < 4 + 4 * nq) {
             const int x = (warp - 4) >> 2;
             const int r = row0 + x * kTileM + ((warp & 3) << 5) + lane;
@@ -222,7 +274,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         return;
     }
 
-    // ---- setup: barriers, TMEM ----
+    // ---- setup: barriers, TMEM; the producer starts loading before the CTA-wide sync ----
+    // K/V ring entry k (K_j0, V_j0, K_j0+1, V_j0+1, ...): one tile of 32 KB into stage k % kStages
+    auto issue_kv = [&](int k) {
+        const int stage = k % kStages;
+        const int j = w.j0 + (k >> 1);
+        const CUtensorMap* map = (k & 1) ? &tm_v : &tm_k;
+        const uint32_t dst = smem_base + kSmemKVOff + stage * kTileBytes;
+        const uint32_t bar = bar_kv_full + 8 * stage;
+        ptx::mbar_expect_tx(bar, kTileBytes);
+        if (!PAGED) {
+            ptx::tma_load_3d(dst, map, bar, 0, j * kTileN, w.g);
+            ptx::tma_load_3d(dst + kHalfBytes, map, bar, 64, j * kTileN, w.g);
+        } else {
+            // two 64-token pages per tile; a tile that ends in the episode's last page
+            // re-reads that page for its second half (masked, but finite)
+            const int npages = (w.L + w.n + 63) >> 6;
+            const int p0 = 2 * j;
+            const int p1 = (p0 + 1 < npages) ? p0 + 1 : p0;
+            const int* pt = a.page_table + (long)w.b * a.max_pages;
+            const int pg0 = pt[p0], pg1 = pt[p1];
+            ptx::tma_load_4d(dst, map, bar, 0, 0, w.g, pg0);
+            ptx::tma_load_4d(dst + 8192, map, bar, 0, 0, w.g, pg1);
+            ptx::tma_load_4d(dst + kHalfBytes, map, bar, 64, 0, w.g, pg0);
+            ptx::tma_load_4d(dst + kHalfBytes + 8192, map, bar, 64, 0, w.g, pg1);
+        }
+    };
+    const int kv_total = 2 * ntiles;
+    const int kv_early = kv_total < kStages ? kv_total : kStages;   // entries that need no free-stage wait
+
+    if (threadIdx.x == 32) {
+        ptx::prefetch_tensormap(&tm_q);
+        ptx::prefetch_tensormap(&tm_k);
+        ptx::prefetch_tensormap(&tm_v);
+    }
     if (threadIdx.x == 0) {
         ptx::mbar_init(bar_q_full, 1);
         ptx::mbar_init(bar_q_full + 8, 1);
@@ -237,9 +322,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         *s_abort = 0;
         ptx::fence_barrier_init();
-        ptx::prefetch_tensormap(&tm_q);
-        ptx::prefetch_tensormap(&tm_k);
-        ptx::prefetch_tensormap(&tm_v);
+        // everything this CTA reads or writes in global memory follows this thread's loads, so one
+        // wait here orders the whole CTA after the kernels it depends on
+        ptx::grid_dependency_wait();
+        // first loads go out now: they only need the barriers this thread has just initialised
+        const int qrow = w.row_base + row0;
+        for (int x = 0; x < nq; ++x) {
+            const uint32_t dst = smem_base + kSmemQOff + x * kTileBytes;
+            ptx::mbar_expect_tx(bar_q_full + 8 * x, kTileBytes);
+            ptx::tma_load_3d(dst, &tm_q, bar_q_full + 8 * x, 0, qrow + x * kTileM, w.g);
+            ptx::tma_load_3d(dst + kHalfBytes, &tm_q, bar_q_full + 8 * x, 64, qrow + x * kTileM, w.g);
+            if (x == 0) issue_kv(0);
+        }
+        for (int k = 1; k < kv_early; ++k) issue_kv(k);
     }
     if (warp == 1) {
         ptx::tmem_alloc(tmem_slot, 512);
@@ -249,50 +344,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __syncthreads();
     ptx::fence_after_sync();
     const uint32_t tmem = *s_tmem;
+    ptx::grid_launch_dependents();
     if (threadIdx.x == 0) EVLN_STAMP(1);
 
+    // register budget: the producer / MMA warpgroup gives registers to the softmax warpgroups,
+    // which hold a whole 128-column score row per thread
+    if (warp < 4) ptx::setmaxnreg_dec<80>();
+
     if (warp == 0) {
-        // ================= TMA producer =================
-        bool ok = true;
-        int issued = 0;
+        // ================= TMA producer (remaining ring entries) =================
         if (lane == 0) {
-            const int qrow = w.row_base + row0;
-            for (int x = 0; x < nq; ++x) {
-                const uint32_t dst = smem_base + kSmemQOff + x * kTileBytes;
-                ptx::mbar_expect_tx(bar_q_full + 8 * x, kTileBytes);
-                ptx::tma_load_3d(dst, &tm_q, bar_q_full + 8 * x, 0, qrow + x * kTileM, w.g);
-                ptx::tma_load_3d(dst + kHalfBytes, &tm_q, bar_q_full + 8 * x, 64, qrow + x * kTileM, w.g);
-            }
-            const int total = 2 * ntiles;          // K_j0, V_j0, K_j0+1, V_j0+1, ...
-            for (int k = 0; k < total && ok; ++k) {
+            bool ok = true;
+            int issued = kv_early;
+            for (int k = kv_early; k < kv_total; ++k) {
                 const int stage = k % kStages;
                 const uint32_t parity = ((k / kStages) & 1) ^ 1;
                 ok = wait_bounded(bar_kv_empty + 8 * stage, parity, kDevTimeoutProducer, a.status, s_abort);
                 if (!ok) break;
-                const int j = w.j0 + (k >> 1);
-                const CUtensorMap* map = (k & 1) ? &tm_v : &tm_k;
-                const uint32_t dst = smem_base + kSmemKVOff + stage * kTileBytes;
-                const uint32_t bar = bar_kv_full + 8 * stage;
-                ptx::mbar_expect_tx(bar, kTileBytes);
-                if (!PAGED) {
-                    ptx::tma_load_3d(dst, map, bar, 0, j * kTileN, w.g);
-                    ptx::tma_load_3d(dst + kHalfBytes, map, bar, 64, j * kTileN, w.g);
-                } else {
-                    // two 64-token pages per tile; a tile that ends in the episode's last page
-                    // re-reads that page for its second half (masked, but finite)
-                    const int npages = (w.L + w.n + 63) >> 6;
-                    const int p0 = 2 * j;
-                    const int p1 = (p0 + 1 < npages) ? p0 + 1 : p0;
-                    const int* pt = a.page_table + (long)w.b * a.max_pages;
-                    const int pg0 = pt[p0], pg1 = pt[p1];
-                    ptx::tma_load_4d(dst, map, bar, 0, 0, w.g, pg0);
-                    ptx::tma_load_4d(dst + 8192, map, bar, 0, 0, w.g, pg1);
-                    ptx::tma_load_4d(dst + kHalfBytes, map, bar, 64, 0, w.g, pg0);
-                    ptx::tma_load_4d(dst + kHalfBytes + 8192, map, bar, 64, 0, w.g, pg1);
-                }
+                issue_kv(k);
                 ++issued;
             }
-            if (!ok) {
+            if (!ok || *s_abort) {
                 // drain: every load this thread issued must have landed before the CTA may exit
                 for (int k = (issued > kStages ? issued - kStages : 0); k < issued; ++k) {
                     const int stage = k % kStages;
@@ -313,33 +385,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
         // every wait is taken by the whole warp and its outcome made uniform
         auto wait_u = [&](uint32_t bar, uint32_t parity, int code) -> bool {
-            const bool r = wait_bounded(bar, parity, code, a.status, s_abort);
-            return __all_sync(0xffffffffu, r);
+            return warp_wait(bar, parity, code, a.status, s_abort, lane);
         };
         auto wait_kv = [&](int kk) -> bool {
             return wait_u(bar_kv_full + 8 * (kk % kStages), (kk / kStages) & 1, kDevTimeoutMmaKV);
         };
+        // descriptors differ only in their address field (units of 16 bytes): build them once
+        const uint64_t qdesc0 = make_sdesc(smem_base + kSmemQOff, 16, 1024);
+        const uint64_t kdesc0 = make_sdesc(smem_base + kSmemKVOff, 16, 1024);            // K-major
+        const uint64_t vdesc0 = make_sdesc(smem_base + kSmemKVOff, kHalfBytes, 1024);    // MN-major
         auto issue_s = [&](int x, int kk) {      // S_x = Q_x K^T, K in ring entry kk
             if (lane == 0) {
-                const uint32_t qa = smem_base + kSmemQOff + x * kTileBytes;
-                const uint32_t kb = smem_base + kSmemKVOff + (kk % kStages) * kTileBytes;
+                const uint64_t qd = qdesc0 + (uint64_t)((x * kTileBytes) >> 4);
+                const uint64_t kd = kdesc0 + (uint64_t)(((kk % kStages) * kTileBytes) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    ptx::mma_ss(tmem + kColS + x * 128, make_sdesc(qa + off, 16, 1024),
-                                make_sdesc(kb + off, 16, 1024), idesc_s, ks > 0);
+                    const uint64_t off = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                    ptx::mma_ss(tmem + kColS + x * 128, qd + off, kd + off, idesc_s, ks > 0);
                 }
                 ptx::mma_commit(bar_s_full + 8 * x);
             }
         };
         auto issue_pv = [&](int x, int kk, bool accumulate) {   // O_x (+)= P_x V, V in ring entry kk
             if (lane == 0) {
-                const uint32_t vb = smem_base + kSmemKVOff + (kk % kStages) * kTileBytes;
+                const uint64_t vd = vdesc0 + (uint64_t)(((kk % kStages) * kTileBytes) >> 4);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     ptx::mma_ts(tmem + kColO + x * 128, tmem + kColS + x * 128 + ks * 8,
-                                make_sdesc(vb + ks * 2048, kHalfBytes, 1024), idesc_pv,
-                                accumulate || ks > 0);
+                                vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, accumulate || ks > 0);
                 }
             }
         };
@@ -368,6 +441,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (x < nq && ok) {
                     ok = wait_u(bar_p_full + 8 * x, p_parity, kDevTimeoutMmaP);
                     if (ok) {
+                        if (lane == 0 && it < 6) EVLN_STAMP(32 + 4 * it + 2 * x);
                         ptx::fence_after_sync();
                         issue_pv(x, kv, it > 0);
                         if (more) {
@@ -379,6 +453,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                             release(kv);
                             if (more) release(kn);
                         }
+                        if (lane == 0 && it < 6) EVLN_STAMP(33 + 4 * it + 2 * x);
                         __syncwarp();
                     }
                 }
@@ -387,6 +462,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
     } else if (warp >= 4 && warp < 4 + 4 * nq) {
         // ================= softmax + epilogue =================
+        ptx::setmaxnreg_inc<208>();
         const int x = (warp - 4) >> 2;                     // which query tile
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
         const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
@@ -400,11 +476,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         float m_ref = -INFINITY;      // reference maximum (log2 domain) the exponentials use
         float l = 0.f;                // running sum of exponentials
         bool ok = true;
-        uint32_t regs[32];
+        const uint64_t scale2 = ptx::pack2(a.scale_log2, a.scale_log2);
 
         for (int it = 0; it < ntiles; ++it) {
-            ok = wait_bounded(bar_s_full + 8 * x, it & 1, kDevTimeoutSoftmaxS, a.status, s_abort);
-            ok = __all_sync(0xffffffffu, ok);
+            ok = warp_wait(bar_s_full + 8 * x, it & 1, kDevTimeoutSoftmaxS, a.status, s_abort, lane);
             if (!ok) break;
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(2 + 2 * it);
@@ -413,22 +488,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             const int lim = bound - j * kTileN;            // columns 0..lim are visible
             const bool no_mask = __all_sync(0xffffffffu, lim >= kTileN - 1);
 
-            // pass 1: row maximum of the visible scores
-            float tmax = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                ptx::tmem_ld32(t_s + c * 32, regs);
-                ptx::tmem_ld_wait();
-                if (no_mask) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(regs[e]));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (c * 32 + e <= lim) tmax = fmaxf(tmax, __uint_as_float(regs[e]));
-                }
+            // the whole score row of this thread: 128 columns in registers, one wait
+            uint32_t sA[32], sB[32], sC[32], sD[32];
+            ptx::tmem_ld32(t_s, sA);
+            ptx::tmem_ld32(t_s + 32, sB);
+            ptx::tmem_ld32(t_s + 64, sC);
+            ptx::tmem_ld32(t_s + 96, sD);
+            ptx::tmem_ld_wait();
+            if (warp == 4 && lane == 0 && it < 6) EVLN_STAMP(14 + 2 * it);
+            if (!no_mask) {        // -inf: masked keys (and stale slots) drop out
+                mask32(sA, lim);
+                mask32(sB, lim - 32);
+                mask32(sC, lim - 64);
+                mask32(sD, lim - 96);
             }
-            tmax *= a.scale_log2;                           // scale > 0: max commutes with it
+
+            // row maximum (3-input max, four independent chains)
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            rowmax32(sA, mx0, mx1, mx2, mx3);
+            rowmax32(sB, mx0, mx1, mx2, mx3);
+            rowmax32(sC, mx0, mx1, mx2, mx3);
+            rowmax32(sD, mx0, mx1, mx2, mx3);
+            const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
 
             // move the reference maximum only when it would otherwise lose range
             float alpha = 1.f;
@@ -440,6 +521,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             if (it > 0 && __any_sync(0xffffffffu, grow)) {
                 // O_x holds PV sums up to tile it-1 (complete: the S commit follows them)
+                uint32_t regs[32];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     ptx::tmem_ld32(t_o + c * 32, regs);
@@ -450,28 +532,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
             }
 
-            // pass 2: P = 2^(s*scale_log2 - m_ref), row sum, bf16 P over the S columns
+            if (warp == 4 && lane == 0 && it < 6) EVLN_STAMP(15 + 2 * it);
+            // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P over the S columns
             const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            float lsum = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                ptx::tmem_ld32(t_s + c * 32, regs);
-                ptx::tmem_ld_wait();
-                uint32_t packed[16];
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float p0 = ptx::ex2(fmaf(__uint_as_float(regs[e]), a.scale_log2, neg_m));
-                    float p1 = ptx::ex2(fmaf(__uint_as_float(regs[e + 1]), a.scale_log2, neg_m));
-                    if (!no_mask) {
-                        if (c * 32 + e > lim) p0 = 0.f;
-                        if (c * 32 + e + 1 > lim) p1 = 0.f;
-                    }
-                    lsum += p0 + p1;
-                    packed[e >> 1] = ptx::pack_bf16x2(p0, p1);
-                }
-                ptx::tmem_st16(t_s + c * 16, packed);
+            const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
+            uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
+            exp32_store(sA, t_s, scale2, negm2, sum2a, sum2b);
+            exp32_store(sB, t_s + 16, scale2, negm2, sum2a, sum2b);
+            exp32_store(sC, t_s + 32, scale2, negm2, sum2a, sum2b);
+            exp32_store(sD, t_s + 48, scale2, negm2, sum2a, sum2b);
+            {
+                float a0, a1, b0, b1;
+                ptx::unpack2(sum2a, a0, a1);
+                ptx::unpack2(sum2b, b0, b1);
+                l += (a0 + a1) + (b0 + b1);
             }
-            l += lsum;
             ptx::tmem_st_wait();
             ptx::fence_before_sync();
             ptx::mbar_arrive(bar_p_full + 8 * x);
@@ -479,30 +554,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
 
         if (ok) {
-            ok = wait_bounded(bar_o_full + 8 * x, 0, kDevTimeoutSoftmaxO, a.status, s_abort);
-            ok = __all_sync(0xffffffffu, ok);
+            ok = warp_wait(bar_o_full + 8 * x, 0, kDevTimeoutSoftmaxO, a.status, s_abort, lane);
         }
         if (ok) {
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(28);
+            // Epilogue: O/l goes out through shared memory so that global stores are whole
+            // 128-byte lines.  This tile's Q buffer is dead (its last S MMA has completed); each
+            // warp stages its own 32 rows there, 32 channels at a time, rows 144 bytes apart.
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
-            const long prow = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + r_local;
-            float4* dst = reinterpret_cast<float4*>(a.o_part + prow * 128);
+            const int wrow0 = quarter << 5;
+            uint8_t* stage = smem_gen + kSmemQOff + x * kTileBytes + wrow0 * 144;
+            const int first_row = row0 + x * kTileM + wrow0;                 // episode-local
+            const int rows_here = rows_valid - first_row;                    // may be <= 0 or > 32
+            const long prow0 = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + first_row;
+            float* gbase = a.o_part + prow0 * 128;
+            uint32_t regs[32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 ptx::tmem_ld32(t_o + c * 32, regs);
                 ptx::tmem_ld_wait();
-                if (row_valid) {
+                float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        dst[c * 8 + (e >> 2)] = make_float4(__uint_as_float(regs[e]) * inv,
-                                                            __uint_as_float(regs[e + 1]) * inv,
-                                                            __uint_as_float(regs[e + 2]) * inv,
-                                                            __uint_as_float(regs[e + 3]) * inv);
+                for (int e = 0; e < 32; e += 4)
+                    srow[e >> 2] = make_float4(__uint_as_float(regs[e]) * inv, __uint_as_float(regs[e + 1]) * inv,
+                                               __uint_as_float(regs[e + 2]) * inv, __uint_as_float(regs[e + 3]) * inv);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = i * 4 + (lane >> 3);
+                    if (r < rows_here) {
+                        const float4 v = *reinterpret_cast<const float4*>(stage + r * 144 + (lane & 7) * 16);
+                        *reinterpret_cast<float4*>(gbase + (long)r * 128 + c * 32 + (lane & 7) * 4) = v;
+                    }
                 }
+                __syncwarp();
             }
             if (row_valid)
-                a.lse_part[prow] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                a.lse_part[prow0 + lane] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
             if (warp == 4 && lane == 0) EVLN_STAMP(29);
         }
     }

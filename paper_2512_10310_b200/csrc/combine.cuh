@@ -29,6 +29,8 @@ __global__ void __launch_bounds__(128)
 combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
 {
     constexpr int C = D / 32;
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long row = (long)blockIdx.x * 4 + warp;      // packed row within kv head
     const int g = blockIdx.y;

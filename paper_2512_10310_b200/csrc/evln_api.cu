@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include <new>
+#include <utility>
 
 #include "attn_simt.cuh"
 #include "attn_tcgen05.cuh"
@@ -37,6 +38,26 @@ extern "C" void evlnDebugSetTimeline(void* p) { g_timeline = (long long*)p; }
 #endif
 
 namespace {
+
+// Every kernel is launched with programmatic stream serialisation: its prologue may overlap the
+// tail of the previous kernel in the stream; each kernel waits (griddepcontrol.wait) before it
+// touches global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -192,12 +213,12 @@ evlnStatus_t launch_combine(evlnHandle_t h, const CombineArgs& a, int D, bool pa
 {
     dim3 grid(ceil_div(a.rows, 4), a.Hkv);
     if (paged) {
-        if (D == 128) combine_kernel<T, 128, true, BatchLens><<<grid, 128, 0, st>>>(a, *bl);
+        if (D == 128) launch_pdl(combine_kernel<T, 128, true, BatchLens>, dim3(grid), dim3(128), 0, st, a, *bl);
         else return EVLN_NOT_SUPPORTED;
     } else {
         NoLens nl = {};
-        if (D == 128) combine_kernel<T, 128, false, NoLens><<<grid, 128, 0, st>>>(a, nl);
-        else combine_kernel<T, 64, false, NoLens><<<grid, 128, 0, st>>>(a, nl);
+        if (D == 128) launch_pdl(combine_kernel<T, 128, false, NoLens>, dim3(grid), dim3(128), 0, st, a, nl);
+        else launch_pdl(combine_kernel<T, 64, false, NoLens>, dim3(grid), dim3(128), 0, st, a, nl);
     }
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
@@ -338,9 +359,9 @@ evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void*
     NoLens nl = {};
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16)
-        rope_append_kernel<__nv_bfloat16, false, NoLens><<<p->num_new, 256, 0, st>>>(a, nl);
+        launch_pdl(rope_append_kernel<__nv_bfloat16, false, NoLens>, dim3(p->num_new), dim3(256), 0, st, a, nl);
     else
-        rope_append_kernel<float, false, NoLens><<<p->num_new, 256, 0, st>>>(a, nl);
+        launch_pdl(rope_append_kernel<float, false, NoLens>, dim3(p->num_new), dim3(256), 0, st, a, nl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
@@ -392,7 +413,7 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
 #endif
         NoLens nl = {};
         const int grid = S * p->num_kv_heads * a.units_per_head;
-        attn_tc_kernel<false, NoLens><<<grid, kTcThreads, kTcSmemBytes, st>>>(tm_q, tm_k, tm_v, a, nl);
+        launch_pdl(attn_tc_kernel<false, NoLens>, dim3(grid), dim3(kTcThreads), kTcSmemBytes, st, tm_q, tm_k, tm_v, a, nl);
     } else {
         SimtAttnArgs a = {};
         a.q_rot = q_rot; a.k_cache = k_cache; a.v_cache = v_cache;
@@ -402,11 +423,11 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
         a.num_splits = S; a.scale = scale;
         dim3 grid(ceil_div(R, 4), p->num_kv_heads, S);
         if (p->dtype == EVLN_BF16) {
-            if (D == 128) attn_simt_kernel<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(a);
-            else attn_simt_kernel<__nv_bfloat16, 64><<<grid, 128, 0, st>>>(a);
+            if (D == 128) launch_pdl(attn_simt_kernel<__nv_bfloat16, 128>, dim3(grid), dim3(128), 0, st, a);
+            else launch_pdl(attn_simt_kernel<__nv_bfloat16, 64>, dim3(grid), dim3(128), 0, st, a);
         } else {
-            if (D == 128) attn_simt_kernel<float, 128><<<grid, 128, 0, st>>>(a);
-            else attn_simt_kernel<float, 64><<<grid, 128, 0, st>>>(a);
+            if (D == 128) launch_pdl(attn_simt_kernel<float, 128>, dim3(grid), dim3(128), 0, st, a);
+            else launch_pdl(attn_simt_kernel<float, 64>, dim3(grid), dim3(128), 0, st, a);
         }
     }
     cudaError_t e = cudaGetLastError();
@@ -471,7 +492,7 @@ evlnStatus_t evlnPagedRopeAppend(evlnHandle_t h, const evlnPagedParams* p, const
     a.log2_theta = log2(p->rope_theta);
     BatchLens bl;
     fill_lens(&bl, p, h_cache_lens, h_new_offsets);
-    rope_append_kernel<__nv_bfloat16, true, BatchLens><<<total, 256, 0, (cudaStream_t)stream>>>(a, bl);
+    launch_pdl(rope_append_kernel<__nv_bfloat16, true, BatchLens>, dim3(total), dim3(256), 0, (cudaStream_t)stream, a, bl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
@@ -520,8 +541,7 @@ evlnStatus_t evlnPagedStepAttention(evlnHandle_t h, const evlnPagedParams* p, co
     a.scale_log2 = scale * 1.4426950408889634f;
     BatchLens bl;
     fill_lens(&bl, p, h_cache_lens, h_new_offsets);
-    attn_tc_kernel<true, BatchLens><<<(int)items, kTcThreads, kTcSmemBytes, (cudaStream_t)stream>>>(
-        tm_q, tm_k, tm_v, a, bl);
+    launch_pdl(attn_tc_kernel<true, BatchLens>, dim3((int)items), dim3(kTcThreads), kTcSmemBytes, (cudaStream_t)stream, tm_q, tm_k, tm_v, a, bl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }

@@ -37,6 +37,8 @@ __global__ void __launch_bounds__(256)
 rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
 {
     constexpr int V = VecTraits<T>::kVec;
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ double s_cos[128];
     __shared__ double s_sin[128];
 
