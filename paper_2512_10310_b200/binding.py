@@ -15,7 +15,7 @@ from ctypes import (POINTER, Structure, byref, c_char_p, c_double, c_float, c_in
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "lib", "libevln.so")
-_SOURCES = ["evln_api.cu", "attn_tcgen05.cuh", "attn_simt.cuh", "combine.cuh", "rope_append.cuh",
+_SOURCES = ["evln_api.cu", "attn_pair.cuh", "attn_simt.cuh", "combine.cuh", "rope_append.cuh",
             "common.cuh", "ptx_sm100.cuh"]
 
 EVLN_OK, EVLN_INVALID_VALUE, EVLN_NOT_SUPPORTED, EVLN_CACHE_FULL = 0, 1, 2, 3

@@ -1,0 +1,668 @@
+// Split-KV step attention on the 5th-generation tensor cores, one CTA pair per work item
+// (bf16, head_dim 128).
+//
+// Sec. 3.2 leaves one attention per step: the n new (rotated) queries against all L+n cached
+// keys.  With grouped-query attention the G query heads of a kv head share its K/V, so the
+// G*n query rows of a kv head are packed row-major (row = token*G + head-in-group) and cut
+// into 128-row tiles.  A UNIT is two consecutive tiles (256 rows); a work item is a unit and a
+// contiguous range of 128-key KV tiles (a split).  A cluster of two CTAs owns a work item: CTA
+// r of the pair holds query tile r, and both drive ONE tensor-core instruction stream
+// (tcgen05.mma cta_group::2, M = 256) issued by the pair's CTA 0.  Each CTA stages only its
+// half of every K tile (64 keys) and V tile (64 channels): the pair reads K/V once for 256
+// query rows.  The item's normalised partial outputs + log-sum-exps go to the workspace that
+// the combine kernel merges.
+//
+// Per CTA (384 threads, 1 CTA/SM, ~197 KB shared memory, all 512 TMEM columns):
+//   warp 0      TMA producer: the CTA's Q tile once, then its K / V half tiles through two
+//               5-deep rings of 16 KB stages (128B-swizzled); no multicast anywhere.  Bytes are
+//               counted on barriers of CTA 0, where the MMA thread waits.
+//   warp 1      (CTA 0) MMA issuer, one lane: S_j = Q K_j^T (SS) into one of THREE score
+//               buffers, O += P_j V_j (A = P from TMEM).  Scores run up to three tiles ahead
+//               of the softmax, so the tensor pipe and the softmax warps only meet through
+//               full/empty barriers and neither waits for the other's latency.
+//   warps 4-11  softmax + epilogue: thread (row, half) owns 64 of the 128 score columns of a
+//               row; the two threads of a row agree on the row maximum through shared memory
+//               once per tile, off the critical path: the exponentials are taken against the
+//               row's current reference while the exchange is in flight and redone only if the
+//               reference has to move.  P is written back over the scores as packed bf16; O is
+//               rescaled in TMEM only when the row maximum grew by more than 2^8 (the final
+//               division by the row sum makes that exact).
+//   warps 2-3   idle.
+// TMEM columns: S_b at 128*b, b = 0..2; P_b (packed bf16) sits in columns [0,32) and [64,96) of S_b,
+// each half over the score columns of the thread that writes it; O at 384.
+//
+// Every mbarrier wait is bounded: on expiry the CTA records a code in the device status word and
+// raises a shared abort flag; all roles then leave their loops, TMEM is freed and the pair
+// returns together (cluster barrier).
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx_sm100.cuh"
+
+namespace evln {
+
+#ifdef EVLN_TIMELINE
+#define EVLN_STAMP(slot) do { if (a.timeline && (slot) < 64) a.timeline[(long)blockIdx.x * 64 + (slot)] = clock64(); } while (0)
+#else
+#define EVLN_STAMP(slot) do { } while (0)
+#endif
+
+constexpr int kTcThreads = 384;
+constexpr int kKStages = 5, kVStages = 5;
+constexpr int kTileBytes = kTileM * 128 * 2;          // Q tile: 128 rows x 128 channels x bf16
+constexpr int kHalfBytes = kTileBytes / 2;            // 16 KB: a 64-channel half of Q; a K or V half tile
+constexpr int kSmemQOff = 0;
+constexpr int kSmemKOff = kTileBytes;
+constexpr int kSmemVOff = kSmemKOff + kKStages * kHalfBytes;
+constexpr int kSmemBarOff = kSmemVOff + kVStages * kHalfBytes;
+constexpr int kSmemBarBytes = 320;
+constexpr int kSmemXchOff = kSmemBarOff + kSmemBarBytes;          // float [2 parities][2 halves][128 rows]
+constexpr int kSmemXchBytes = 2 * 2 * 128 * 4;
+constexpr int kTcSmemBytes = kSmemXchOff + kSmemXchBytes + 1024;  // + slack to align to 1024
+constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at boost clocks
+constexpr int kScoreBufs = 3;
+constexpr uint32_t kColO = 384;
+constexpr float kGrowLimit = 8.f;                     // log2 headroom before a row's reference moves
+
+struct TcAttnArgs {
+    float* o_part;            // [S, Hkv, rows, 128]
+    float* lse_part;          // [S, Hkv, rows]
+    const int* page_table;    // paged only
+    int* status;              // device status word
+    int Hkv, G;
+    int rows;                 // packed rows per kv head over the whole call
+    int cache_len, num_new;   // contiguous only
+    int num_splits;           // contiguous only
+    int units_per_head;       // contiguous only
+    int batch, max_pages, chunk_tiles;   // paged only
+    float scale_log2;         // softmax scale * log2(e)
+#ifdef EVLN_TIMELINE
+    long long* timeline;      // debug builds only: 64 clock stamps per CTA
+#endif
+};
+
+// --- descriptors --------------------------------------------------------------------------
+
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, M x N of the whole pair.
+__device__ __forceinline__ constexpr uint32_t make_idesc(bool b_mn_major, int m, int n)
+{
+    return (1u << 4)                       // D format: f32
+           | (1u << 7)                     // A format: bf16
+           | (1u << 10)                    // B format: bf16
+           | ((b_mn_major ? 1u : 0u) << 16)
+           | ((uint32_t)(n >> 3) << 17)
+           | ((uint32_t)(m >> 4) << 24);
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;                // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                // SWIZZLE_128B
+    return d;
+}
+
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, int code, int* status,
+                                             volatile int* s_abort)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3f) == 0) {
+            if (*s_abort) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *s_abort = 1;
+                atomicCAS(status, 0, code);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// One lane polls, the warp shares the outcome (fewer pollers on the barrier word).
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, int code, int* status,
+                                          volatile int* s_abort, int lane)
+{
+    int r = 1;
+    if (lane == 0) r = wait_bounded(bar, parity, code, status, s_abort) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, r, 0) != 0;
+}
+
+// --- softmax pieces on one 32-column register block of a score row ---------------------------
+
+__device__ __forceinline__ void mask32(uint32_t (&s)[32], int lim)
+{
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+        if (e > lim) s[e] = 0xff800000u;
+}
+
+__device__ __forceinline__ void rowmax32(const uint32_t (&s)[32], float& m0, float& m1, float& m2, float& m3)
+{
+#pragma unroll
+    for (int e = 0; e < 32; e += 8) {
+        m0 = ptx::max3(m0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+        m1 = ptx::max3(m1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+        m2 = ptx::max3(m2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+        m3 = ptx::max3(m3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
+    }
+}
+
+// p = 2^(s*scale + negm) for 32 columns, accumulated into two packed sums, written to TMEM as
+// 16 columns of packed bf16 pairs
+__device__ __forceinline__ void exp32_store(const uint32_t (&s)[32], uint32_t taddr, uint64_t scale2,
+                                            uint64_t negm2, uint64_t& sum2a, uint64_t& sum2b)
+{
+    uint32_t packed[16];
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        const uint64_t xa = ptx::fma2(ptx::pack2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), scale2, negm2);
+        const uint64_t xb = ptx::fma2(ptx::pack2(__uint_as_float(s[e + 2]), __uint_as_float(s[e + 3])), scale2, negm2);
+        float x0, x1, x2, x3;
+        ptx::unpack2(xa, x0, x1);
+        ptx::unpack2(xb, x2, x3);
+        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1), p2 = ptx::ex2(x2), p3 = ptx::ex2(x3);
+        sum2a = ptx::add2(sum2a, ptx::pack2(p0, p1));
+        sum2b = ptx::add2(sum2b, ptx::pack2(p2, p3));
+        packed[e >> 1] = ptx::pack_bf16x2(p0, p1);
+        packed[(e >> 1) + 1] = ptx::pack_bf16x2(p2, p3);
+    }
+    ptx::tmem_st16(taddr, packed);
+}
+
+// --- work decoding ------------------------------------------------------------------------
+
+struct WorkItem {
+    int b, g, unit, slot;     // episode, kv head, unit within the episode, partial slot
+    int L, n;                 // episode lengths
+    int row_base;             // first packed row of the episode within the kv head
+    int j0, j1;               // KV tile range
+};
+
+template <bool PAGED, typename LensT>
+__device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT& lens, int item)
+{
+    WorkItem w;
+    if (!PAGED) {
+        w.b = 0;
+        w.unit = item % a.units_per_head;
+        w.g = (item / a.units_per_head) % a.Hkv;
+        w.slot = item / (a.units_per_head * a.Hkv);
+        w.L = a.cache_len;
+        w.n = a.num_new;
+        w.row_base = 0;
+        const int nkv = unit_kv_tiles(w.L, w.n, a.G, w.unit, kUnitRows);
+        w.j0 = (int)((long)w.slot * nkv / a.num_splits);
+        w.j1 = (int)((long)(w.slot + 1) * nkv / a.num_splits);
+    } else {
+        int rem = item;
+        int b = 0;
+        for (; b < a.batch; ++b) {
+            const int n_b = lens.new_off[b + 1] - lens.new_off[b];
+            const int units = ceil_div(n_b * a.G, kUnitRows);
+            int per_head = 0;
+            for (int u = 0; u < units; ++u)
+                per_head += ceil_div(unit_kv_tiles(lens.cache_len[b], n_b, a.G, u, kUnitRows), a.chunk_tiles);
+            if (rem < per_head * a.Hkv) {
+                w.b = b;
+                w.L = lens.cache_len[b];
+                w.n = n_b;
+                w.row_base = lens.new_off[b] * a.G;
+                w.g = rem / per_head;
+                rem -= w.g * per_head;
+                for (int u = 0; u < units; ++u) {
+                    const int nkv = unit_kv_tiles(w.L, n_b, a.G, u, kUnitRows);
+                    const int S = ceil_div(nkv, a.chunk_tiles);
+                    if (rem < S) {
+                        w.unit = u;
+                        w.slot = rem;
+                        w.j0 = (int)((long)rem * nkv / S);
+                        w.j1 = (int)((long)(rem + 1) * nkv / S);
+                        break;
+                    }
+                    rem -= S;
+                }
+                break;
+            }
+            rem -= per_head * a.Hkv;
+        }
+        if (b == a.batch) { w.b = -1; w.j0 = w.j1 = 0; w.g = w.unit = w.slot = 0; w.L = w.n = w.row_base = 0; }
+    }
+    return w;
+}
+
+// --- the kernel ---------------------------------------------------------------------------
+// Launched with a cluster of 2 CTAs along x: work item = blockIdx.x / 2, query tile = rank.
+
+template <bool PAGED, typename LensT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const TcAttnArgs a,
+                 const __grid_constant__ LensT lens)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+
+    // barriers: same offsets in both CTAs; "(CTA 0)" marks those of which only CTA 0's copy is used
+    const uint32_t bar_base = smem_base + kSmemBarOff;
+    const uint32_t bar_q_full = bar_base;                        // (CTA 0) both CTAs' Q tiles landed
+    const uint32_t bar_k_full = bar_q_full + 8;                  // (CTA 0) [kKStages]
+    const uint32_t bar_v_full = bar_k_full + 8 * kKStages;       // (CTA 0) [kVStages]
+    const uint32_t bar_k_empty = bar_v_full + 8 * kVStages;      // [kKStages] stage consumed by the MMAs
+    const uint32_t bar_v_empty = bar_k_empty + 8 * kKStages;     // [kVStages]
+    const uint32_t bar_s_full = bar_v_empty + 8 * kVStages;      // [kScoreBufs] scores ready
+    const uint32_t bar_p_full = bar_s_full + 8 * kScoreBufs;     // (CTA 0) [kScoreBufs] P written by both CTAs
+    const uint32_t bar_pv_done = bar_p_full + 8 * kScoreBufs;    // [2] PV of an even / odd tile landed
+    const uint32_t bar_o_full = bar_pv_done + 16;                // last PV landed
+    const uint32_t bar_xch = bar_o_full + 8;                     // [4] the two warps of a lane quarter meet here
+    const uint32_t tmem_slot = bar_xch + 32;                     // uint32
+    static_assert(8 * (1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 3 + 4) + 8 <= kSmemBarBytes, "barrier area");
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem_gen + (tmem_slot - smem_base) + 4);
+    float* s_xch = reinterpret_cast<float*>(smem_gen + kSmemXchOff);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();      // 0: issues the MMAs, owns the "(CTA 0)" barriers
+    if (threadIdx.x == 0) EVLN_STAMP(0);
+
+    const WorkItem w = decode_work<PAGED, LensT>(a, lens, blockIdx.x >> 1);
+    if (PAGED && w.b < 0) return;                      // both CTAs of the pair decode the same item
+
+    const int rows_valid = w.n * a.G;                            // packed rows of this episode
+    const int row0 = w.unit * kUnitRows + (int)rank * kTileM;    // first row of this CTA's tile (episode-local)
+    const int ntiles = w.j1 - w.j0;
+
+    // A split with no KV tiles (more splits than tiles): its partials are "empty".
+    if (ntiles <= 0) {
+        ptx::grid_dependency_wait();
+        if (warp >= 4 && warp < 8) {
+            const int r = row0 + ((warp & 3) << 5) + lane;
+            if (r < rows_valid) {
+                const long prow = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + r;
+                float4* o = reinterpret_cast<float4*>(a.o_part + prow * 128);
+                for (int c = 0; c < 32; ++c) o[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                a.lse_part[prow] = -INFINITY;
+            }
+        }
+        return;
+    }
+
+    // ---- setup: barriers, TMEM, then the pair synchronises once ----
+    if (threadIdx.x == 32) {
+        ptx::prefetch_tensormap(&tm_q);
+        ptx::prefetch_tensormap(&tm_k);
+        ptx::prefetch_tensormap(&tm_v);
+    }
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(bar_q_full, 2);
+        for (int s = 0; s < kKStages; ++s) {
+            ptx::mbar_init(bar_k_full + 8 * s, 2);
+            ptx::mbar_init(bar_k_empty + 8 * s, 1);
+        }
+        for (int s = 0; s < kVStages; ++s) {
+            ptx::mbar_init(bar_v_full + 8 * s, 2);
+            ptx::mbar_init(bar_v_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < kScoreBufs; ++b) {
+            ptx::mbar_init(bar_s_full + 8 * b, 1);
+            ptx::mbar_init(bar_p_full + 8 * b, 16);      // 8 softmax warps in each CTA
+        }
+        ptx::mbar_init(bar_pv_done, 1);
+        ptx::mbar_init(bar_pv_done + 8, 1);
+        ptx::mbar_init(bar_o_full, 1);
+        for (int q = 0; q < 4; ++q) ptx::mbar_init(bar_xch + 8 * q, 2);
+        *s_abort = 0;
+        ptx::fence_barrier_init();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(tmem_slot, 512);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::fence_before_sync();
+    __syncthreads();
+    ptx::cluster_arrive();      // the other CTA's barriers exist before anything arrives on them
+    ptx::cluster_wait();
+    ptx::fence_after_sync();
+    const uint32_t tmem = *s_tmem;
+    ptx::grid_launch_dependents();
+    if (threadIdx.x == 0) EVLN_STAMP(1);
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            // everything this CTA reads or writes in global memory follows this thread's loads, so
+            // one wait here orders the whole CTA after the kernels it depends on
+            ptx::grid_dependency_wait();
+            const uint32_t q_full0 = ptx::map_to_cta(bar_q_full, 0);
+            {
+                const uint32_t dst = smem_base + kSmemQOff;
+                const int qrow = w.row_base + row0;
+                ptx::mbar_expect_tx_cluster(q_full0, kTileBytes);
+                ptx::tma_load_3d_pair(dst, &tm_q, q_full0, 0, qrow, w.g);
+                ptx::tma_load_3d_pair(dst + kHalfBytes, &tm_q, q_full0, 64, qrow, w.g);
+            }
+            bool ok = true;
+            // this CTA's half of K tile j: keys [128 j + 64 rank, +64), all channels (two 64-channel blocks)
+            auto load_k = [&](int jj) {
+                const int stage = jj % kKStages;
+                if (jj >= kKStages)
+                    ok = wait_bounded(bar_k_empty + 8 * stage, ((jj / kKStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
+                if (!ok) return;
+                const uint32_t dst = smem_base + kSmemKOff + stage * kHalfBytes;
+                const uint32_t bar = ptx::map_to_cta(bar_k_full + 8 * stage, 0);
+                const int j = w.j0 + jj;
+                ptx::mbar_expect_tx_cluster(bar, kHalfBytes);
+                if (!PAGED) {
+                    const int key0 = j * kTileN + (int)rank * 64;
+                    ptx::tma_load_3d_pair(dst, &tm_k, bar, 0, key0, w.g);
+                    ptx::tma_load_3d_pair(dst + 8192, &tm_k, bar, 64, key0, w.g);
+                } else {
+                    // a 64-token page is exactly this CTA's half; past the episode's last page the
+                    // last page is read again (masked, but finite)
+                    const int npages = (w.L + w.n + 63) >> 6;
+                    int pi = 2 * j + (int)rank;
+                    if (pi >= npages) pi = npages - 1;
+                    const int pg = a.page_table[(long)w.b * a.max_pages + pi];
+                    ptx::tma_load_4d_pair(dst, &tm_k, bar, 0, 0, w.g, pg);
+                    ptx::tma_load_4d_pair(dst + 8192, &tm_k, bar, 64, 0, w.g, pg);
+                }
+            };
+            // this CTA's half of V tile j: all 128 keys, channels [64 rank, +64)
+            auto load_v = [&](int jj) {
+                const int stage = jj % kVStages;
+                if (jj >= kVStages)
+                    ok = wait_bounded(bar_v_empty + 8 * stage, ((jj / kVStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
+                if (!ok) return;
+                const uint32_t dst = smem_base + kSmemVOff + stage * kHalfBytes;
+                const uint32_t bar = ptx::map_to_cta(bar_v_full + 8 * stage, 0);
+                const int j = w.j0 + jj;
+                ptx::mbar_expect_tx_cluster(bar, kHalfBytes);
+                if (!PAGED) {
+                    ptx::tma_load_3d_pair(dst, &tm_v, bar, 64 * (int)rank, j * kTileN, w.g);
+                } else {
+                    const int npages = (w.L + w.n + 63) >> 6;
+                    const int p0 = 2 * j;
+                    const int p1 = (p0 + 1 < npages) ? p0 + 1 : p0;
+                    const int* pt = a.page_table + (long)w.b * a.max_pages;
+                    ptx::tma_load_4d_pair(dst, &tm_v, bar, 64 * (int)rank, 0, w.g, pt[p0]);
+                    ptx::tma_load_4d_pair(dst + 8192, &tm_v, bar, 64 * (int)rank, 0, w.g, pt[p1]);
+                }
+            };
+            // in the order the MMAs consume them: K_0..K_2, then V_j, K_{j+3}
+            const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
+            for (int jj = 0; jj < pre && ok; ++jj) load_k(jj);
+            for (int jj = 0; jj < ntiles && ok; ++jj) {
+                load_v(jj);
+                if (ok && jj + kScoreBufs < ntiles) load_k(jj + kScoreBufs);
+            }
+            if (!ok || *s_abort) {
+                // give this CTA's loads in flight time to land before the pair may leave
+                const long long t0 = clock64();
+                while (clock64() - t0 < 400000) { }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1 && rank == 0) {
+        // ================= MMA issuer (CTA 0 of the pair) =================
+        const uint32_t idesc_s = make_idesc(false, 2 * kTileM, kTileN);
+        const uint32_t idesc_pv = make_idesc(true, 2 * kTileM, 128);
+        const uint16_t both = 3;
+        bool ok = true;
+        auto wait_u = [&](uint32_t bar, uint32_t parity, int code) -> bool {
+            return warp_wait(bar, parity, code, a.status, s_abort, lane);
+        };
+        // descriptors differ only in their address field (units of 16 bytes): build them once
+        const uint64_t qdesc0 = make_sdesc(smem_base + kSmemQOff, 16, 1024);
+        const uint64_t kdesc0 = make_sdesc(smem_base + kSmemKOff, 16, 1024);            // K-major, 64 keys per CTA
+        const uint64_t vdesc0 = make_sdesc(smem_base + kSmemVOff, kHalfBytes, 1024);    // MN-major, 64 channels per CTA
+        auto issue_s = [&](int jj) {             // S_jj = Q K_jj^T into score buffer jj % 3
+            if (lane == 0) {
+                const int stage = jj % kKStages;
+                const uint64_t kd = kdesc0 + (uint64_t)((stage * kHalfBytes) >> 4);
+                const uint32_t d = tmem + (uint32_t)(jj % kScoreBufs) * 128;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t qoff = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
+                    const uint64_t koff = (uint64_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4);
+                    ptx::mma_ss_pair(d, qdesc0 + qoff, kd + koff, idesc_s, ks > 0);
+                }
+                ptx::mma_commit_pair(bar_s_full + 8 * (jj % kScoreBufs), both);
+                ptx::mma_commit_pair(bar_k_empty + 8 * stage, both);
+            }
+        };
+        auto issue_pv = [&](int jj) {            // O (+)= P_jj V_jj
+            if (lane == 0) {
+                const int stage = jj % kVStages;
+                const uint64_t vd = vdesc0 + (uint64_t)((stage * kHalfBytes) >> 4);
+                const uint32_t p = tmem + (uint32_t)(jj % kScoreBufs) * 128;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    ptx::mma_ts_pair(tmem + kColO, p + (ks >> 2) * 64 + (ks & 3) * 8, vd + (uint64_t)((ks * 2048) >> 4),
+                                     idesc_pv, jj > 0 || ks > 0);
+                ptx::mma_commit_pair(bar_pv_done + 8 * (jj & 1), both);
+                ptx::mma_commit_pair(bar_v_empty + 8 * stage, both);
+                if (jj == ntiles - 1) ptx::mma_commit_pair(bar_o_full, both);
+            }
+        };
+
+        ok = wait_u(bar_q_full, 0, kDevTimeoutMmaQ);
+        const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
+        for (int jj = 0; jj < pre && ok; ++jj) {
+            ok = wait_u(bar_k_full + 8 * (jj % kKStages), (jj / kKStages) & 1, kDevTimeoutMmaKV);
+            if (ok) {
+                ptx::fence_after_sync();
+                issue_s(jj);
+                __syncwarp();
+            }
+        }
+        for (int jj = 0; jj < ntiles && ok; ++jj) {
+            ok = wait_u(bar_v_full + 8 * (jj % kVStages), (jj / kVStages) & 1, kDevTimeoutMmaKV);
+            if (lane == 0 && jj < 8) EVLN_STAMP(32 + 3 * jj);
+            if (ok) ok = wait_u(bar_p_full + 8 * (jj % kScoreBufs), (jj / kScoreBufs) & 1, kDevTimeoutMmaP);
+            if (!ok) break;
+            if (lane == 0 && jj < 8) EVLN_STAMP(33 + 3 * jj);
+            ptx::fence_after_sync();
+            issue_pv(jj);
+            const int jn = jj + kScoreBufs;
+            if (jn < ntiles) {
+                ok = wait_u(bar_k_full + 8 * (jn % kKStages), (jn / kKStages) & 1, kDevTimeoutMmaKV);
+                if (ok) {
+                    ptx::fence_after_sync();
+                    issue_s(jn);
+                }
+            }
+            if (lane == 0 && jj < 8) EVLN_STAMP(34 + 3 * jj);
+            __syncwarp();
+        }
+    } else if (warp >= 4) {
+        // ================= softmax + epilogue =================
+        const int quarter = warp & 3;                      // TMEM lane quarter of this warp
+        const int half = (warp - 4) >> 2;                  // which 64 columns of a row
+        const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
+        const int r_local = row0 + r_tile;                 // packed row within the episode
+        const bool row_valid = r_local < rows_valid;
+        const int bound = row_valid ? w.L + r_local / a.G : -1;   // last visible key index
+        const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
+        const uint32_t t_o = t_lane + kColO + half * 64;
+        const uint32_t p_full0 = ptx::map_to_cta(bar_p_full, 0);
+
+        float m_ref = -INFINITY;      // reference maximum (log2 domain) the exponentials use
+        float l = 0.f;                // this thread's share of the running sum of exponentials
+        bool ok = true;
+        const uint64_t scale2 = ptx::pack2(a.scale_log2, a.scale_log2);
+        // Meeting number k of the two warps of this lane quarter (one phase of their barrier each):
+        // what either wrote to shared memory before its arrival is visible to the other after the wait.
+        auto meet_arrive = [&]() {
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
+        };
+        auto meet_wait = [&](int k) -> bool {
+            return warp_wait(bar_xch + 8 * quarter, k & 1, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
+        };
+
+        for (int jj = 0; jj < ntiles; ++jj) {
+            const int buf = jj % kScoreBufs;
+            ok = warp_wait(bar_s_full + 8 * buf, (jj / kScoreBufs) & 1, kDevTimeoutSoftmaxS, a.status, s_abort, lane);
+            if (!ok) break;
+            ptx::fence_after_sync();
+            if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(2 + 3 * jj);
+
+            const int lim = bound - (w.j0 + jj) * kTileN - half * 64;   // columns 0..lim of this half are visible
+            const bool no_mask = __all_sync(0xffffffffu, lim >= 63);
+            const uint32_t t_s = t_lane + buf * 128 + half * 64;
+            const uint32_t t_p = t_s;       // P over this thread's own score columns only: nobody else's are touched
+
+            uint32_t sA[32], sB[32];
+            ptx::tmem_ld32(t_s, sA);
+            ptx::tmem_ld32(t_s + 32, sB);
+            ptx::tmem_ld_wait();
+            if (!no_mask) {        // -inf: masked keys (and stale slots) drop out
+                mask32(sA, lim);
+                mask32(sB, lim - 32);
+            }
+
+            // row maximum of this thread's 64 columns goes to the other half's thread
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            rowmax32(sA, mx0, mx1, mx2, mx3);
+            rowmax32(sB, mx0, mx1, mx2, mx3);
+            float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
+            float* xch = s_xch + (jj & 1) * 256;
+            xch[half * 128 + r_tile] = tmax;
+            meet_arrive();
+
+            // While the exchange is in flight: exponentials against the row's current reference.  They
+            // stand unless the reference has to move (always for a row's first visible keys).
+            const bool first = __any_sync(0xffffffffu, row_valid && m_ref == -INFINITY);
+            uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
+            if (!first) {
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;   // -inf: a padding row, all masked
+                const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
+                exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
+                exp32_store(sB, t_p + 16, scale2, negm2, sum2a, sum2b);
+            }
+            ok = meet_wait(jj);
+            if (!ok) break;
+            tmax = fmaxf(tmax, xch[(half ^ 1) * 128 + r_tile]);
+            if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(3 + 3 * jj);
+
+            // move the reference maximum only when it would otherwise lose range; both threads of a
+            // row see the same numbers and take the same decision
+            const bool grow = tmax > m_ref + kGrowLimit;    // also true for the first finite tile
+            const bool any_grow = __any_sync(0xffffffffu, grow);
+            if (first || any_grow) {
+                float alpha = 1.f;
+                if (grow) {
+                    alpha = (m_ref == -INFINITY) ? 0.f : ptx::ex2(m_ref - tmax);
+                    m_ref = tmax;
+                    l *= alpha;
+                }
+                if (jj > 0 && any_grow) {
+                    // O must hold the products up to tile jj-1 before it is rescaled.  PV(jj-3) landed
+                    // before these scores were written, so the barrier of this parity has seen either
+                    // (jj-1)/2 or (jj-1)/2 + 1 phases: the parity test is unambiguous.
+                    ok = warp_wait(bar_pv_done + 8 * ((jj - 1) & 1), ((jj - 1) >> 1) & 1, kDevTimeoutSoftmaxO, a.status,
+                                   s_abort, lane);
+                    if (!ok) break;
+                    ptx::fence_after_sync();
+                    uint32_t regs[32];
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {              // this thread's 64 of the row's 128 channels
+                        ptx::tmem_ld32(t_o + c * 32, regs);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
+                        ptx::tmem_st32(t_o + c * 32, regs);
+                    }
+                }
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
+                sum2a = ptx::pack2(0.f, 0.f);
+                sum2b = sum2a;
+                exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
+                exp32_store(sB, t_p + 16, scale2, negm2, sum2a, sum2b);
+            }
+            {
+                float a0, a1, b0, b1;
+                ptx::unpack2(sum2a, a0, a1);
+                ptx::unpack2(sum2b, b0, b1);
+                l += (a0 + a1) + (b0 + b1);
+            }
+            ptx::tmem_st_wait();
+            ptx::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(p_full0 + 8 * buf);
+            if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(4 + 3 * jj);
+        }
+
+        if (ok) ok = warp_wait(bar_o_full, 0, kDevTimeoutSoftmaxO, a.status, s_abort, lane);
+        if (ok) {
+            ptx::fence_after_sync();
+            if (warp == 4 && lane == 0) EVLN_STAMP(60);
+            // the row sum is the two halves' sums (same reference in both)
+            float* xch = s_xch + (ntiles & 1) * 256;
+            xch[half * 128 + r_tile] = l;
+            meet_arrive();
+            ok = meet_wait(ntiles);
+        }
+        if (ok) {
+            const float* xch = s_xch + (ntiles & 1) * 256;
+            l += xch[(half ^ 1) * 128 + r_tile];
+            // Epilogue: O/l goes out through shared memory so that global stores are whole
+            // 128-byte lines.  The K ring is dead (its last consumer has completed); each warp
+            // stages its 32 rows there, 32 channels at a time, rows 144 bytes apart.
+            const float inv = (l > 0.f) ? 1.f / l : 0.f;
+            const int wrow0 = quarter << 5;
+            uint8_t* stage = smem_gen + kSmemKOff + (warp - 4) * (32 * 144);
+            const int first_row = row0 + wrow0;                              // episode-local
+            const int rows_here = rows_valid - first_row;                    // may be <= 0 or > 32
+            const long prow0 = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + first_row;
+            float* gbase = a.o_part + prow0 * 128 + half * 64;
+            uint32_t regs[32];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                ptx::tmem_ld32(t_o + c * 32, regs);
+                ptx::tmem_ld_wait();
+                float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
+#pragma unroll
+                for (int e = 0; e < 32; e += 4)
+                    srow[e >> 2] = make_float4(__uint_as_float(regs[e]) * inv, __uint_as_float(regs[e + 1]) * inv,
+                                               __uint_as_float(regs[e + 2]) * inv, __uint_as_float(regs[e + 3]) * inv);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = i * 4 + (lane >> 3);
+                    if (r < rows_here) {
+                        const float4 v = *reinterpret_cast<const float4*>(stage + r * 144 + (lane & 7) * 16);
+                        *reinterpret_cast<float4*>(gbase + (long)r * 128 + c * 32 + (lane & 7) * 4) = v;
+                    }
+                }
+                __syncwarp();
+            }
+            if (row_valid && half == 0)
+                a.lse_part[prow0 + lane] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            if (warp == 4 && lane == 0) EVLN_STAMP(61);
+        }
+    }
+
+    // ---- teardown: nobody leaves while the other CTA may still touch this CTA's memory ----
+    ptx::fence_before_sync();
+    __syncthreads();
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+    if (warp == 1) {
+        ptx::fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem, 512);
+        if (lane == 0) EVLN_STAMP(62);
+    }
+}
+
+}  // namespace evln

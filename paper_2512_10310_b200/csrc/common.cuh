@@ -23,6 +23,7 @@ enum DeviceStatus : int {
     kDevTimeoutMmaP = 4,       // MMA warp waiting for the softmax warps' P tile
     kDevTimeoutSoftmaxS = 5,   // softmax warps waiting for S
     kDevTimeoutSoftmaxO = 6,   // softmax warps waiting for the final O
+    kDevTimeoutSoftmaxX = 7,   // softmax warps of one lane quarter waiting for each other
 };
 
 // Per-episode lengths of a paged batch, passed by value.

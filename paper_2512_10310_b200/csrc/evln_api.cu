@@ -12,7 +12,7 @@
 #include <utility>
 
 #include "attn_simt.cuh"
-#include "attn_tcgen05.cuh"
+#include "attn_pair.cuh"
 #include "combine.cuh"
 #include "common.cuh"
 #include "rope_append.cuh"
@@ -59,6 +59,27 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// The attention kernel runs as clusters of two CTAs (one CTA pair per work item).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pair_pdl(void (*kernel)(KArgs...), int items, size_t smem, cudaStream_t st, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * items);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int elem_bytes(int dtype) { return dtype == EVLN_BF16 ? 2 : 4; }
@@ -91,16 +112,17 @@ inline bool use_tensor_kernel(const evlnStepParams* p)
     return p->kernel == EVLN_KERNEL_AUTO && p->dtype == EVLN_BF16 && p->head_dim == 128;
 }
 
-// Cost model of the split-KV schedule of the tensor-core kernel: `ctas` CTAs run in waves of
-// one per SM, each walks ceil(nkv / S) KV tiles plus a fixed prologue/epilogue; every extra
-// split adds combine traffic.
+// Cost model of the split-KV schedule of the tensor-core kernel: work items (unit x split) run
+// in waves of one CTA pair per two SMs, each walks ceil(nkv / S) KV tiles plus a fixed
+// prologue/epilogue; every extra split adds combine traffic.
 int choose_splits_tc(int units_total, int nkv_max, int nkv_min, int num_sms)
 {
     int best = 1;
     double best_cost = 1e30;
+    const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
     const int smax = nkv_min < kMaxSplits ? (nkv_min < 1 ? 1 : nkv_min) : kMaxSplits;
     for (int s = 1; s <= smax; ++s) {
-        const double waves = ceil((double)units_total * s / num_sms);
+        const double waves = ceil((double)units_total * s / pairs);
         const double cost = waves * (ceil((double)nkv_max / s) + 2.0) + 0.3 * s;
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
@@ -185,7 +207,8 @@ void paged_schedule(evlnHandle_t h, const evlnPagedParams* p, const int* lens, c
     total *= p->num_kv_heads;
     int chunk = p->kv_chunk_tiles;
     if (chunk <= 0) {
-        chunk = (int)((total + (long)h->num_sms * 4 - 1) / ((long)h->num_sms * 4));
+        const long pairs = h->num_sms / 2 > 0 ? h->num_sms / 2 : 1;
+        chunk = (int)((total + pairs * 4 - 1) / (pairs * 4));
         if (chunk < 8) chunk = 8;
     }
     if (chunk < ceil_div(nkv_max, kMaxSplits)) chunk = ceil_div(nkv_max, kMaxSplits);
@@ -266,10 +289,10 @@ evlnStatus_t evlnCreate(evlnHandle_t* handle, int device)
     e = cudaMalloc(&h->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int));
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(attn_tc_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(attn_pair_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kTcSmemBytes);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(attn_tc_kernel<true, BatchLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(attn_pair_kernel<true, BatchLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kTcSmemBytes);
     if (e != cudaSuccess) {
         if (h->d_status) cudaFree(h->d_status);
@@ -398,9 +421,12 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
             // rows past L+n read as zeros, so stale slots never reach the tensor core
             cuuint64_t dims[3] = {128, (cuuint64_t)T, (cuuint64_t)p->num_kv_heads};
             cuuint64_t strides[2] = {256, (cuuint64_t)p->cache_capacity * 256};
-            cuuint32_t box[3] = {64, 128, 1};
-            if (!encode_map(h, &tm_k, k_cache, 3, dims, strides, box)) return EVLN_INVALID_VALUE;
-            if (!encode_map(h, &tm_v, v_cache, 3, dims, strides, box)) return EVLN_INVALID_VALUE;
+            // per CTA of a pair: half a K tile is 64 keys x all channels (two boxes), half a V tile
+            // is 128 keys x 64 channels (one box)
+            cuuint32_t box_k[3] = {64, 64, 1};
+            cuuint32_t box_v[3] = {64, 128, 1};
+            if (!encode_map(h, &tm_k, k_cache, 3, dims, strides, box_k)) return EVLN_INVALID_VALUE;
+            if (!encode_map(h, &tm_v, v_cache, 3, dims, strides, box_v)) return EVLN_INVALID_VALUE;
         }
         TcAttnArgs a = {};
         a.o_part = o_part; a.lse_part = lse_part; a.page_table = nullptr; a.status = h->d_status;
@@ -412,8 +438,8 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
         a.timeline = g_timeline;
 #endif
         NoLens nl = {};
-        const int grid = S * p->num_kv_heads * a.units_per_head;
-        launch_pdl(attn_tc_kernel<false, NoLens>, dim3(grid), dim3(kTcThreads), kTcSmemBytes, st, tm_q, tm_k, tm_v, a, nl);
+        const int items = S * p->num_kv_heads * a.units_per_head;
+        launch_pair_pdl(attn_pair_kernel<false, NoLens>, items, kTcSmemBytes, st, tm_q, tm_k, tm_v, a, nl);
     } else {
         SimtAttnArgs a = {};
         a.q_rot = q_rot; a.k_cache = k_cache; a.v_cache = v_cache;
@@ -515,7 +541,7 @@ evlnStatus_t evlnPagedStepAttention(evlnHandle_t h, const evlnPagedParams* p, co
     long items;
     paged_schedule(h, p, h_cache_lens, h_new_offsets, &chunk, &smax, &items);
     if (workspace_bytes < partial_bytes(smax, p->num_kv_heads, rows, 128)) return EVLN_WORKSPACE_TOO_SMALL;
-    if (items <= 0 || items > 0x7fffffffL) return EVLN_NOT_SUPPORTED;
+    if (items <= 0 || items > 0x3fffffffL) return EVLN_NOT_SUPPORTED;
 
     CUtensorMap tm_q, tm_k, tm_v;
     {
@@ -541,7 +567,7 @@ evlnStatus_t evlnPagedStepAttention(evlnHandle_t h, const evlnPagedParams* p, co
     a.scale_log2 = scale * 1.4426950408889634f;
     BatchLens bl;
     fill_lens(&bl, p, h_cache_lens, h_new_offsets);
-    launch_pdl(attn_tc_kernel<true, BatchLens>, dim3((int)items), dim3(kTcThreads), kTcSmemBytes, (cudaStream_t)stream, tm_q, tm_k, tm_v, a, bl);
+    launch_pair_pdl(attn_pair_kernel<true, BatchLens>, (int)items, kTcSmemBytes, (cudaStream_t)stream, tm_q, tm_k, tm_v, a, bl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
@@ -611,7 +637,7 @@ evlnStatus_t noalloc_setup(int device, NoAllocDevice** out)
         cudaDriverEntryPointQueryResult qres;
         e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
         if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return EVLN_CUDA_ERROR;
-        e = cudaFuncSetAttribute(attn_tc_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(attn_pair_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kTcSmemBytes);
         if (e != cudaSuccess) return EVLN_CUDA_ERROR;
         d->ctx.device = device;
