@@ -16,7 +16,7 @@
 //   warp 0      TMA producer: the CTA's Q tile once, then its K / V half tiles through two
 //               5-deep rings of 16 KB stages (128B-swizzled); no multicast anywhere.  Bytes are
 //               counted on barriers of CTA 0, where the MMA thread waits.
-//   warp 1      (CTA 0) MMA issuer, one lane: S_j = Q K_j^T (SS) into one of THREE score
+//   warp 1      (CTA 0) MMA issuer, one elected lane: S_j = Q K_j^T (SS) into one of THREE score
 //               buffers, O += P_j V_j (A = P from TMEM).  Scores run up to three tiles ahead
 //               of the softmax, so the tensor pipe and the softmax warps only meet through
 //               full/empty barriers and neither waits for the other's latency.
@@ -425,7 +425,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint64_t kdesc0 = make_sdesc(smem_base + kSmemKOff, 16, 1024);            // K-major, 64 keys per CTA
         const uint64_t vdesc0 = make_sdesc(smem_base + kSmemVOff, kHalfBytes, 1024);    // MN-major, 64 channels per CTA
         auto issue_s = [&](int jj) {             // S_jj = Q K_jj^T into score buffer jj % 3
-            if (lane == 0) {
+            if (ptx::elect_one()) {
                 const int stage = jj % kKStages;
                 const uint64_t kd = kdesc0 + (uint64_t)((stage * kHalfBytes) >> 4);
                 const uint32_t d = tmem + (uint32_t)(jj % kScoreBufs) * 128;
@@ -440,7 +440,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
         };
         auto issue_pv = [&](int jj) {            // O (+)= P_jj V_jj
-            if (lane == 0) {
+            if (ptx::elect_one()) {
                 const int stage = jj % kVStages;
                 const uint64_t vd = vdesc0 + (uint64_t)((stage * kHalfBytes) >> 4);
                 const uint32_t p = tmem + (uint32_t)(jj % kScoreBufs) * 128;
