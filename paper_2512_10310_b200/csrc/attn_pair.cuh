@@ -12,7 +12,7 @@
 // query rows.  The item's normalised partial outputs + log-sum-exps go to the workspace that
 // the combine kernel merges.
 //
-// Per CTA (384 threads, 1 CTA/SM, ~197 KB shared memory, all 512 TMEM columns):
+// Per CTA (640 threads, 1 CTA/SM, ~199 KB shared memory, all 512 TMEM columns):
 //   warp 0      TMA producer: the CTA's Q tile once, then its K / V half tiles through two
 //               5-deep rings of 16 KB stages (128B-swizzled); no multicast anywhere.  Bytes are
 //               counted on barriers of CTA 0, where the MMA thread waits.
@@ -20,16 +20,18 @@
 //               buffers, O += P_j V_j (A = P from TMEM).  Scores run up to three tiles ahead
 //               of the softmax, so the tensor pipe and the softmax warps only meet through
 //               full/empty barriers and neither waits for the other's latency.
-//   warps 4-11  softmax + epilogue: thread (row, half) owns 64 of the 128 score columns of a
-//               row; the two threads of a row agree on the row maximum through shared memory
-//               once per tile, off the critical path: the exponentials are taken against the
-//               row's current reference while the exchange is in flight and redone only if the
-//               reference has to move.  P is written back over the scores as packed bf16; O is
-//               rescaled in TMEM only when the row maximum grew by more than 2^8 (the final
-//               division by the row sum makes that exact).
+//   warps 4-19  softmax + epilogue: thread (row, part) owns 32 of the 128 score columns of a
+//               row, so every SM sub-partition has four softmax warps whose barrier, TMEM and
+//               special-function latencies (each 100-200 cycles) hide one another.  The four
+//               threads of a row agree on the row maximum through shared memory once per tile,
+//               off the critical path: the exponentials are taken against the row's current
+//               reference while the exchange is in flight and redone only if the reference has
+//               to move.  P is written back over the scores as packed bf16; O is rescaled in
+//               TMEM only when the row maximum grew by more than 2^8 (the final division by the
+//               row sum makes that exact).
 //   warps 2-3   idle.
-// TMEM columns: S_b at 128*b, b = 0..2; P_b (packed bf16) sits in columns [0,32) and [64,96) of S_b,
-// each half over the score columns of the thread that writes it; O at 384.
+// TMEM columns: S_b at 128*b, b = 0..2; P_b (packed bf16) sits in columns [32c, 32c+16), c = 0..3,
+// of S_b, each part over the score columns of the thread that writes it; O at 384.
 //
 // Every mbarrier wait is bounded: on expiry the CTA records a code in the device status word and
 // raises a shared abort flag; all roles then leave their loops, TMEM is freed and the pair
@@ -49,7 +51,8 @@ namespace evln {
 #define EVLN_STAMP(slot) do { } while (0)
 #endif
 
-constexpr int kTcThreads = 384;
+constexpr int kTcThreads = 640;
+constexpr int kParts = 4;                             // threads per score row (32 columns each)
 constexpr int kKStages = 5, kVStages = 5;
 constexpr int kTileBytes = kTileM * 128 * 2;          // Q tile: 128 rows x 128 channels x bf16
 constexpr int kHalfBytes = kTileBytes / 2;            // 16 KB: a 64-channel half of Q; a K or V half tile
@@ -58,8 +61,8 @@ constexpr int kSmemKOff = kTileBytes;
 constexpr int kSmemVOff = kSmemKOff + kKStages * kHalfBytes;
 constexpr int kSmemBarOff = kSmemVOff + kVStages * kHalfBytes;
 constexpr int kSmemBarBytes = 320;
-constexpr int kSmemXchOff = kSmemBarOff + kSmemBarBytes;          // float [2 parities][2 halves][128 rows]
-constexpr int kSmemXchBytes = 2 * 2 * 128 * 4;
+constexpr int kSmemXchOff = kSmemBarOff + kSmemBarBytes;          // float [2 parities][kParts][128 rows]
+constexpr int kSmemXchBytes = 2 * kParts * 128 * 4;
 constexpr int kTcSmemBytes = kSmemXchOff + kSmemXchBytes + 1024;  // + slack to align to 1024
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at boost clocks
 constexpr int kScoreBufs = 3;
@@ -263,7 +266,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const uint32_t bar_p_full = bar_s_full + 8 * kScoreBufs;     // (CTA 0) [kScoreBufs] P written by both CTAs
     const uint32_t bar_pv_done = bar_p_full + 8 * kScoreBufs;    // [2] PV of an even / odd tile landed
     const uint32_t bar_o_full = bar_pv_done + 16;                // last PV landed
-    const uint32_t bar_xch = bar_o_full + 8;                     // [4] the two warps of a lane quarter meet here
+    const uint32_t bar_xch = bar_o_full + 8;                     // [4] the kParts warps of a lane quarter meet here
     const uint32_t tmem_slot = bar_xch + 32;                     // uint32
     static_assert(8 * (1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 3 + 4) + 8 <= kSmemBarBytes, "barrier area");
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
@@ -314,12 +317,12 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
         for (int b = 0; b < kScoreBufs; ++b) {
             ptx::mbar_init(bar_s_full + 8 * b, 1);
-            ptx::mbar_init(bar_p_full + 8 * b, 16);      // 8 softmax warps in each CTA
+            ptx::mbar_init(bar_p_full + 8 * b, 8 * kParts);      // 4 * kParts softmax warps in each CTA
         }
         ptx::mbar_init(bar_pv_done, 1);
         ptx::mbar_init(bar_pv_done + 8, 1);
         ptx::mbar_init(bar_o_full, 1);
-        for (int q = 0; q < 4; ++q) ptx::mbar_init(bar_xch + 8 * q, 2);
+        for (int q = 0; q < 4; ++q) ptx::mbar_init(bar_xch + 8 * q, kParts);
         *s_abort = 0;
         ptx::fence_barrier_init();
     }
@@ -446,7 +449,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const uint32_t p = tmem + (uint32_t)(jj % kScoreBufs) * 128;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    ptx::mma_ts_pair(tmem + kColO, p + (ks >> 2) * 64 + (ks & 3) * 8, vd + (uint64_t)((ks * 2048) >> 4),
+                    ptx::mma_ts_pair(tmem + kColO, p + (ks >> 1) * 32 + (ks & 1) * 8, vd + (uint64_t)((ks * 2048) >> 4),
                                      idesc_pv, jj > 0 || ks > 0);
                 ptx::mma_commit_pair(bar_pv_done + 8 * (jj & 1), both);
                 ptx::mma_commit_pair(bar_v_empty + 8 * stage, both);
@@ -465,48 +468,55 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
         }
         for (int jj = 0; jj < ntiles && ok; ++jj) {
-            ok = wait_u(bar_v_full + 8 * (jj % kVStages), (jj / kVStages) & 1, kDevTimeoutMmaKV);
-            if (lane == 0 && jj < 8) EVLN_STAMP(32 + 3 * jj);
-            if (ok) ok = wait_u(bar_p_full + 8 * (jj % kScoreBufs), (jj / kScoreBufs) & 1, kDevTimeoutMmaP);
+            // V_jj, P_jj and K_{jj+3}: a wait costs ~150 cycles even on a completed barrier, so three
+            // lanes take one each and the latencies overlap
+            const int jn = jj + kScoreBufs;
+            {
+                uint32_t bar = bar_v_full + 8 * (jj % kVStages), parity = (jj / kVStages) & 1;
+                int code = kDevTimeoutMmaKV;
+                if (lane == 1) { bar = bar_p_full + 8 * (jj % kScoreBufs); parity = (jj / kScoreBufs) & 1; code = kDevTimeoutMmaP; }
+                if (lane == 2) { bar = bar_k_full + 8 * (jn % kKStages); parity = (jn / kKStages) & 1; }
+                bool mine = true;
+                if (lane < 2 || (lane == 2 && jn < ntiles)) mine = wait_bounded(bar, parity, code, a.status, s_abort);
+                ok = __all_sync(0xffffffffu, mine);
+            }
             if (!ok) break;
             if (lane == 0 && jj < 8) EVLN_STAMP(33 + 3 * jj);
             ptx::fence_after_sync();
             issue_pv(jj);
-            const int jn = jj + kScoreBufs;
-            if (jn < ntiles) {
-                ok = wait_u(bar_k_full + 8 * (jn % kKStages), (jn / kKStages) & 1, kDevTimeoutMmaKV);
-                if (ok) {
-                    ptx::fence_after_sync();
-                    issue_s(jn);
-                }
-            }
+            if (jn < ntiles) issue_s(jn);
             if (lane == 0 && jj < 8) EVLN_STAMP(34 + 3 * jj);
             __syncwarp();
         }
     } else if (warp >= 4) {
         // ================= softmax + epilogue =================
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
-        const int half = (warp - 4) >> 2;                  // which 64 columns of a row
+        const int part = (warp - 4) >> 2;                  // which 32 columns of a row
         const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
         const int r_local = row0 + r_tile;                 // packed row within the episode
         const bool row_valid = r_local < rows_valid;
         const int bound = row_valid ? w.L + r_local / a.G : -1;   // last visible key index
         const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
-        const uint32_t t_o = t_lane + kColO + half * 64;
+        const uint32_t t_o = t_lane + kColO + part * 32;
         const uint32_t p_full0 = ptx::map_to_cta(bar_p_full, 0);
 
         float m_ref = -INFINITY;      // reference maximum (log2 domain) the exponentials use
         float l = 0.f;                // this thread's share of the running sum of exponentials
         bool ok = true;
         const uint64_t scale2 = ptx::pack2(a.scale_log2, a.scale_log2);
-        // Meeting number k of the two warps of this lane quarter (one phase of their barrier each):
-        // what either wrote to shared memory before its arrival is visible to the other after the wait.
+        // Meeting number k of the kParts warps of this lane quarter (one phase of their barrier each):
+        // what any of them wrote to shared memory before its arrival is visible to the others after the wait.
         auto meet_arrive = [&]() {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
         };
         auto meet_wait = [&](int k) -> bool {
             return warp_wait(bar_xch + 8 * quarter, k & 1, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
+        };
+        auto row_exchange_max = [&](const float* xch, float v) -> float {
+#pragma unroll
+            for (int c = 0; c < kParts; ++c) v = fmaxf(v, xch[c * 128 + r_tile]);
+            return v;
         };
 
         for (int jj = 0; jj < ntiles; ++jj) {
@@ -516,27 +526,22 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(2 + 3 * jj);
 
-            const int lim = bound - (w.j0 + jj) * kTileN - half * 64;   // columns 0..lim of this half are visible
-            const bool no_mask = __all_sync(0xffffffffu, lim >= 63);
-            const uint32_t t_s = t_lane + buf * 128 + half * 64;
+            const int lim = bound - (w.j0 + jj) * kTileN - part * 32;   // columns 0..lim of this part are visible
+            const bool no_mask = __all_sync(0xffffffffu, lim >= 31);
+            const uint32_t t_s = t_lane + buf * 128 + part * 32;
             const uint32_t t_p = t_s;       // P over this thread's own score columns only: nobody else's are touched
 
-            uint32_t sA[32], sB[32];
+            uint32_t sA[32];
             ptx::tmem_ld32(t_s, sA);
-            ptx::tmem_ld32(t_s + 32, sB);
             ptx::tmem_ld_wait();
-            if (!no_mask) {        // -inf: masked keys (and stale slots) drop out
-                mask32(sA, lim);
-                mask32(sB, lim - 32);
-            }
+            if (!no_mask) mask32(sA, lim);  // -inf: masked keys (and stale slots) drop out
 
-            // row maximum of this thread's 64 columns goes to the other half's thread
+            // row maximum of this thread's 32 columns goes to the row's other threads
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
             rowmax32(sA, mx0, mx1, mx2, mx3);
-            rowmax32(sB, mx0, mx1, mx2, mx3);
             float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
-            float* xch = s_xch + (jj & 1) * 256;
-            xch[half * 128 + r_tile] = tmax;
+            float* xch = s_xch + (jj & 1) * (kParts * 128);
+            xch[part * 128 + r_tile] = tmax;
             meet_arrive();
 
             // While the exchange is in flight: exponentials against the row's current reference.  They
@@ -547,14 +552,13 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;   // -inf: a padding row, all masked
                 const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
                 exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
-                exp32_store(sB, t_p + 16, scale2, negm2, sum2a, sum2b);
             }
             ok = meet_wait(jj);
             if (!ok) break;
-            tmax = fmaxf(tmax, xch[(half ^ 1) * 128 + r_tile]);
+            tmax = row_exchange_max(xch, tmax);
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(3 + 3 * jj);
 
-            // move the reference maximum only when it would otherwise lose range; both threads of a
+            // move the reference maximum only when it would otherwise lose range; all threads of a
             // row see the same numbers and take the same decision
             const bool grow = tmax > m_ref + kGrowLimit;    // also true for the first finite tile
             const bool any_grow = __any_sync(0xffffffffu, grow);
@@ -573,22 +577,18 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                                    s_abort, lane);
                     if (!ok) break;
                     ptx::fence_after_sync();
-                    uint32_t regs[32];
+                    uint32_t regs[32];              // this thread's 32 of the row's 128 channels
+                    ptx::tmem_ld32(t_o, regs);
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {              // this thread's 64 of the row's 128 channels
-                        ptx::tmem_ld32(t_o + c * 32, regs);
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
-                        ptx::tmem_st32(t_o + c * 32, regs);
-                    }
+                    for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
+                    ptx::tmem_st32(t_o, regs);
                 }
                 const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
                 const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
                 sum2a = ptx::pack2(0.f, 0.f);
                 sum2b = sum2a;
                 exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
-                exp32_store(sB, t_p + 16, scale2, negm2, sum2a, sum2b);
             }
             {
                 float a0, a1, b0, b1;
@@ -607,47 +607,45 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (ok) {
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(60);
-            // the row sum is the two halves' sums (same reference in both)
-            float* xch = s_xch + (ntiles & 1) * 256;
-            xch[half * 128 + r_tile] = l;
+            // the row sum is the sum over the row's threads (same reference in all)
+            float* xch = s_xch + (ntiles & 1) * (kParts * 128);
+            xch[part * 128 + r_tile] = l;
             meet_arrive();
             ok = meet_wait(ntiles);
         }
         if (ok) {
-            const float* xch = s_xch + (ntiles & 1) * 256;
-            l += xch[(half ^ 1) * 128 + r_tile];
+            const float* xch = s_xch + (ntiles & 1) * (kParts * 128);
+            l = 0.f;
+#pragma unroll
+            for (int c = 0; c < kParts; ++c) l += xch[c * 128 + r_tile];
             // Epilogue: O/l goes out through shared memory so that global stores are whole
             // 128-byte lines.  The K ring is dead (its last consumer has completed); each warp
-            // stages its 32 rows there, 32 channels at a time, rows 144 bytes apart.
+            // stages its 32 rows x 32 channels there, rows 144 bytes apart.
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             const int wrow0 = quarter << 5;
             uint8_t* stage = smem_gen + kSmemKOff + (warp - 4) * (32 * 144);
             const int first_row = row0 + wrow0;                              // episode-local
             const int rows_here = rows_valid - first_row;                    // may be <= 0 or > 32
             const long prow0 = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + first_row;
-            float* gbase = a.o_part + prow0 * 128 + half * 64;
+            float* gbase = a.o_part + prow0 * 128 + part * 32;
             uint32_t regs[32];
+            ptx::tmem_ld32(t_o, regs);
+            ptx::tmem_ld_wait();
+            float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                ptx::tmem_ld32(t_o + c * 32, regs);
-                ptx::tmem_ld_wait();
-                float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
+            for (int e = 0; e < 32; e += 4)
+                srow[e >> 2] = make_float4(__uint_as_float(regs[e]) * inv, __uint_as_float(regs[e + 1]) * inv,
+                                           __uint_as_float(regs[e + 2]) * inv, __uint_as_float(regs[e + 3]) * inv);
+            __syncwarp();
 #pragma unroll
-                for (int e = 0; e < 32; e += 4)
-                    srow[e >> 2] = make_float4(__uint_as_float(regs[e]) * inv, __uint_as_float(regs[e + 1]) * inv,
-                                               __uint_as_float(regs[e + 2]) * inv, __uint_as_float(regs[e + 3]) * inv);
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = i * 4 + (lane >> 3);
-                    if (r < rows_here) {
-                        const float4 v = *reinterpret_cast<const float4*>(stage + r * 144 + (lane & 7) * 16);
-                        *reinterpret_cast<float4*>(gbase + (long)r * 128 + c * 32 + (lane & 7) * 4) = v;
-                    }
+            for (int i = 0; i < 8; ++i) {
+                const int r = i * 4 + (lane >> 3);
+                if (r < rows_here) {
+                    const float4 v = *reinterpret_cast<const float4*>(stage + r * 144 + (lane & 7) * 16);
+                    *reinterpret_cast<float4*>(gbase + (long)r * 128 + (lane & 7) * 4) = v;
                 }
-                __syncwarp();
             }
-            if (row_valid && half == 0)
+            if (row_valid && part == 0)
                 a.lse_part[prow0 + lane] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
             if (warp == 4 && lane == 0) EVLN_STAMP(61);
         }
