@@ -23,12 +23,11 @@
 //   warps 4-19  softmax + epilogue: thread (row, part) owns 32 of the 128 score columns of a
 //               row, so every SM sub-partition has four softmax warps whose barrier, TMEM and
 //               special-function latencies (each 100-200 cycles) hide one another.  The four
-//               threads of a row agree on the row maximum through shared memory once per tile,
-//               off the critical path: the exponentials are taken against the row's current
-//               reference while the exchange is in flight and redone only if the reference has
-//               to move.  P is written back over the scores as packed bf16; O is rescaled in
-//               TMEM only when the row maximum grew by more than 2^8 (the final division by the
-//               row sum makes that exact).
+//               threads of a row fix the row's reference maximum together on the first tile and
+//               talk to each other again only if a later score exceeds it by more than 2^64
+//               (then O, the row sums and the pending P tiles are rescaled by a power of two);
+//               the final division by the row sum makes any reference exact.  P is written
+//               back over the scores as packed bf16.
 //   warps 2-3   idle.
 // TMEM columns: S_b at 128*b, b = 0..2; P_b (packed bf16) sits in columns [32c, 32c+16), c = 0..3,
 // of S_b, each part over the score columns of the thread that writes it; O at 384.
@@ -60,14 +59,19 @@ constexpr int kSmemQOff = 0;
 constexpr int kSmemKOff = kTileBytes;
 constexpr int kSmemVOff = kSmemKOff + kKStages * kHalfBytes;
 constexpr int kSmemBarOff = kSmemVOff + kVStages * kHalfBytes;
-constexpr int kSmemBarBytes = 320;
-constexpr int kSmemXchOff = kSmemBarOff + kSmemBarBytes;          // float [2 parities][kParts][128 rows]
-constexpr int kSmemXchBytes = 2 * kParts * 128 * 4;
+constexpr int kSmemBarBytes = 384;
+constexpr int kSmemXchOff = kSmemBarOff + kSmemBarBytes;          // float [2 meetings][kParts][128 rows]
+constexpr int kSmemCandOff = kSmemXchOff + 2 * kParts * 128 * 4;  // float [kParts][128 rows]: reference requests
+constexpr int kSmemReqOff = kSmemCandOff + kParts * 128 * 4;      // int [4] request flags, int [4][kParts] released tiles
+constexpr int kSmemXchBytes = 2 * kParts * 128 * 4 + kParts * 128 * 4 + 128;
 constexpr int kTcSmemBytes = kSmemXchOff + kSmemXchBytes + 1024;  // + slack to align to 1024
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at boost clocks
 constexpr int kScoreBufs = 3;
 constexpr uint32_t kColO = 384;
-constexpr float kGrowLimit = 8.f;                     // log2 headroom before a row's reference moves
+#ifndef EVLN_REF_HEADROOM
+#define EVLN_REF_HEADROOM 64.f
+#endif
+constexpr float kRefHeadroom = EVLN_REF_HEADROOM;     // a row's reference moves when a score exceeds it by 2^64
 
 struct TcAttnArgs {
     float* o_part;            // [S, Hkv, rows, 128]
@@ -264,14 +268,18 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const uint32_t bar_v_empty = bar_k_empty + 8 * kKStages;     // [kVStages]
     const uint32_t bar_s_full = bar_v_empty + 8 * kVStages;      // [kScoreBufs] scores ready
     const uint32_t bar_p_full = bar_s_full + 8 * kScoreBufs;     // (CTA 0) [kScoreBufs] P written by both CTAs
-    const uint32_t bar_pv_done = bar_p_full + 8 * kScoreBufs;    // [2] PV of an even / odd tile landed
-    const uint32_t bar_o_full = bar_pv_done + 16;                // last PV landed
+    const uint32_t bar_pv_done = bar_p_full + 8 * kScoreBufs;    // [4] PV of tile j landed: barrier j % 4
+    const uint32_t bar_o_full = bar_pv_done + 32;                // last PV landed
     const uint32_t bar_xch = bar_o_full + 8;                     // [4] the kParts warps of a lane quarter meet here
-    const uint32_t tmem_slot = bar_xch + 32;                     // uint32
-    static_assert(8 * (1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 3 + 4) + 8 <= kSmemBarBytes, "barrier area");
+    const uint32_t bar_rare = bar_xch + 32;                      // [4] ... and here when a row's reference has to move
+    const uint32_t tmem_slot = bar_rare + 32;                    // uint32
+    static_assert(8 * (1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5 + 8) + 8 <= kSmemBarBytes, "barrier area");
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem_gen + (tmem_slot - smem_base) + 4);
     float* s_xch = reinterpret_cast<float*>(smem_gen + kSmemXchOff);
+    float* s_cand = reinterpret_cast<float*>(smem_gen + kSmemCandOff);
+    volatile int* s_req = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff);        // [4]
+    volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff) + 4;    // [4][kParts]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();      // 0: issues the MMAs, owns the "(CTA 0)" barriers
@@ -319,10 +327,13 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::mbar_init(bar_s_full + 8 * b, 1);
             ptx::mbar_init(bar_p_full + 8 * b, 8 * kParts);      // 4 * kParts softmax warps in each CTA
         }
-        ptx::mbar_init(bar_pv_done, 1);
-        ptx::mbar_init(bar_pv_done + 8, 1);
         ptx::mbar_init(bar_o_full, 1);
-        for (int q = 0; q < 4; ++q) ptx::mbar_init(bar_xch + 8 * q, kParts);
+        for (int q = 0; q < 4; ++q) {
+            ptx::mbar_init(bar_pv_done + 8 * q, 1);
+            ptx::mbar_init(bar_xch + 8 * q, kParts);
+            ptx::mbar_init(bar_rare + 8 * q, kParts);
+            s_req[q] = 0;
+        }
         *s_abort = 0;
         ptx::fence_barrier_init();
     }
@@ -451,7 +462,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 for (int ks = 0; ks < 8; ++ks)
                     ptx::mma_ts_pair(tmem + kColO, p + (ks >> 1) * 32 + (ks & 1) * 8, vd + (uint64_t)((ks * 2048) >> 4),
                                      idesc_pv, jj > 0 || ks > 0);
-                ptx::mma_commit_pair(bar_pv_done + 8 * (jj & 1), both);
+                ptx::mma_commit_pair(bar_pv_done + 8 * (jj & 3), both);
                 ptx::mma_commit_pair(bar_v_empty + 8 * stage, both);
                 if (jj == ntiles - 1) ptx::mma_commit_pair(bar_o_full, both);
             }
@@ -504,24 +515,124 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         float l = 0.f;                // this thread's share of the running sum of exponentials
         bool ok = true;
         const uint64_t scale2 = ptx::pack2(a.scale_log2, a.scale_log2);
-        // Meeting number k of the kParts warps of this lane quarter (one phase of their barrier each):
-        // what any of them wrote to shared memory before its arrival is visible to the others after the wait.
-        auto meet_arrive = [&]() {
+        // Meeting of the kParts warps of this lane quarter (one phase of their barrier each): what any
+        // of them wrote to shared memory before its arrival is visible to the others after the wait.
+        auto meet = [&](uint32_t bar, int k) -> bool {
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
+            if (lane == 0) ptx::mbar_arrive(bar + 8 * quarter);
+            return warp_wait(bar + 8 * quarter, k & 1, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
         };
-        auto meet_wait = [&](int k) -> bool {
-            return warp_wait(bar_xch + 8 * quarter, k & 1, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
+        // A wait that gives way when a warp of this lane quarter has asked for a new reference:
+        // 0 = the barrier completed, 1 = a request is pending, 2 = gave up (bounded wait expired).
+        auto wait_or_request = [&](uint32_t bar, uint32_t parity, int code) -> int {
+            int r = 0;
+            if (lane == 0) {
+                if (s_req[quarter]) {
+                    r = 1;
+                } else if (!ptx::mbar_try_wait(bar, parity)) {
+                    const long long t0 = clock64();
+                    uint32_t spins = 0;
+                    while (!ptx::mbar_try_wait(bar, parity)) {
+                        if (s_req[quarter]) { r = 1; break; }
+                        if ((++spins & 0x3f) == 0) {
+                            if (*s_abort) { r = 2; break; }
+                            if (clock64() - t0 > kWaitLimitCycles) {
+                                *s_abort = 1;
+                                atomicCAS(a.status, 0, code);
+                                r = 2;
+                                break;
+                            }
+                        }
+                    }
+                }
+            }
+            return __shfl_sync(0xffffffffu, r, 0);
         };
-        auto row_exchange_max = [&](const float* xch, float v) -> float {
+
+        // The exponentials of a row are taken against a reference m_ref that its kParts threads fix
+        // together on the first tile and then leave alone: the division by the row sum at the end
+        // makes any reference exact, and floating point keeps the relative precision as long as
+        // nothing overflows, i.e. as long as no score exceeds the reference by more than
+        // 2^kRefHeadroom.  So after the first tile the warps of a lane quarter do not talk to each
+        // other at all and drift apart, which is what hides their barrier, TMEM and special-function
+        // latencies behind one another.  A thread that does meet such a score asks for a new
+        // reference: every warp of the quarter comes here at its next tile boundary (or out of a
+        // wait), with `released` = the number of tiles whose P it has handed to the tensor core.
+        // Nothing of a tile is consumed before all its parts are handed over, so the slowest warp
+        // bounds what the accumulator holds; everybody then moves its own state to the new reference
+        // (a power-of-two factor, exact): running sum, its channels of O, and its parts of the P
+        // tiles that are written but not yet consumed.
+        int nrare = 0;                // meetings on bar_rare so far
+        auto move_reference = [&](int released, bool mine, float want) -> bool {
+            s_cand[part * 128 + r_tile] = mine ? want : m_ref;
+            if (lane == 0) s_rel[quarter * kParts + part] = released;
+            __syncwarp();
+            if (lane == 0) s_req[quarter] = 1;
+            if (!meet(bar_rare, nrare++)) return false;
+            int r_min = released;
+            float m_new = m_ref;
 #pragma unroll
-            for (int c = 0; c < kParts; ++c) v = fmaxf(v, xch[c * 128 + r_tile]);
-            return v;
+            for (int c = 0; c < kParts; ++c) {
+                r_min = min(r_min, s_rel[quarter * kParts + c]);
+                m_new = fmaxf(m_new, s_cand[c * 128 + r_tile]);
+            }
+            if (part == 0 && lane == 0) s_req[quarter] = 0;
+            // whole powers of two only, so that what is already rounded stays exact
+            float alpha = 1.f;
+            if (m_new > m_ref) {
+                if (m_ref == -INFINITY) {
+                    alpha = 0.f;
+                } else {
+                    const float steps = ceilf(m_new - m_ref);
+                    m_new = m_ref + steps;
+                    alpha = ptx::ex2(-steps);
+                }
+            }
+            const bool any_change = __any_sync(0xffffffffu, alpha != 1.f);
+            if (any_change) {
+                if (r_min > 0) {
+                    // PV(r_min - 1) must have landed.  The slowest warp saw the scores of tile r_min - 1,
+                    // which were written after PV(r_min - 4): at most three products are outstanding and
+                    // barrier (r_min - 1) % 4 has seen (r_min - 1) / 4 or one more phase.
+                    if (!warp_wait(bar_pv_done + 8 * ((r_min - 1) & 3), ((r_min - 1) >> 2) & 1, kDevTimeoutSoftmaxO, a.status,
+                                   s_abort, lane))
+                        return false;
+                    ptx::fence_after_sync();
+                    uint32_t regs[32];              // this thread's 32 of the row's 128 channels
+                    ptx::tmem_ld32(t_o, regs);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
+                    ptx::tmem_st32(t_o, regs);
+                }
+                for (int t = r_min; t < released; ++t) {    // written, not consumed: at most three tiles
+                    uint32_t pk[16];
+                    const uint32_t t_pt = t_lane + (t % kScoreBufs) * 128 + part * 32;
+                    ptx::tmem_ld16(t_pt, pk);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float lo = __uint_as_float(pk[e] << 16) * alpha;
+                        const float hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
+                        pk[e] = ptx::pack_bf16x2(lo, hi);
+                    }
+                    ptx::tmem_st16(t_pt, pk);
+                }
+                l *= alpha;
+                ptx::tmem_st_wait();
+                ptx::fence_before_sync();
+            }
+            m_ref = m_new;
+            return meet(bar_rare, nrare++);
         };
 
         for (int jj = 0; jj < ntiles; ++jj) {
             const int buf = jj % kScoreBufs;
-            ok = warp_wait(bar_s_full + 8 * buf, (jj / kScoreBufs) & 1, kDevTimeoutSoftmaxS, a.status, s_abort, lane);
+            while (ok) {
+                const int r = wait_or_request(bar_s_full + 8 * buf, (jj / kScoreBufs) & 1, kDevTimeoutSoftmaxS);
+                if (r == 0) break;
+                ok = (r == 1) && move_reference(jj, false, 0.f);
+            }
             if (!ok) break;
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(2 + 3 * jj);
@@ -536,60 +647,32 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::tmem_ld_wait();
             if (!no_mask) mask32(sA, lim);  // -inf: masked keys (and stale slots) drop out
 
-            // row maximum of this thread's 32 columns goes to the row's other threads
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
             rowmax32(sA, mx0, mx1, mx2, mx3);
             float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
-            float* xch = s_xch + (jj & 1) * (kParts * 128);
-            xch[part * 128 + r_tile] = tmax;
-            meet_arrive();
-
-            // While the exchange is in flight: exponentials against the row's current reference.  They
-            // stand unless the reference has to move (always for a row's first visible keys).
-            const bool first = __any_sync(0xffffffffu, row_valid && m_ref == -INFINITY);
-            uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
-            if (!first) {
-                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;   // -inf: a padding row, all masked
-                const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
-                exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
+            if (jj == 0) {
+                // the row's reference: its maximum over the whole first tile (-inf: no visible key yet)
+                s_xch[part * 128 + r_tile] = tmax;
+                ok = meet(bar_xch, 0);
+                if (!ok) break;
+#pragma unroll
+                for (int c = 0; c < kParts; ++c) tmax = fmaxf(tmax, s_xch[c * 128 + r_tile]);
+                m_ref = tmax;
+            } else {
+                bool over = tmax > m_ref + kRefHeadroom;
+                while (ok && __any_sync(0xffffffffu, over)) {
+                    ok = move_reference(jj, over, tmax);
+                    over = tmax > m_ref + kRefHeadroom;
+                }
+                if (!ok) break;
             }
-            ok = meet_wait(jj);
-            if (!ok) break;
-            tmax = row_exchange_max(xch, tmax);
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(3 + 3 * jj);
 
-            // move the reference maximum only when it would otherwise lose range; all threads of a
-            // row see the same numbers and take the same decision
-            const bool grow = tmax > m_ref + kGrowLimit;    // also true for the first finite tile
-            const bool any_grow = __any_sync(0xffffffffu, grow);
-            if (first || any_grow) {
-                float alpha = 1.f;
-                if (grow) {
-                    alpha = (m_ref == -INFINITY) ? 0.f : ptx::ex2(m_ref - tmax);
-                    m_ref = tmax;
-                    l *= alpha;
-                }
-                if (jj > 0 && any_grow) {
-                    // O must hold the products up to tile jj-1 before it is rescaled.  PV(jj-3) landed
-                    // before these scores were written, so the barrier of this parity has seen either
-                    // (jj-1)/2 or (jj-1)/2 + 1 phases: the parity test is unambiguous.
-                    ok = warp_wait(bar_pv_done + 8 * ((jj - 1) & 1), ((jj - 1) >> 1) & 1, kDevTimeoutSoftmaxO, a.status,
-                                   s_abort, lane);
-                    if (!ok) break;
-                    ptx::fence_after_sync();
-                    uint32_t regs[32];              // this thread's 32 of the row's 128 channels
-                    ptx::tmem_ld32(t_o, regs);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
-                    ptx::tmem_st32(t_o, regs);
-                }
-                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
-                sum2a = ptx::pack2(0.f, 0.f);
-                sum2b = sum2a;
-                exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
-            }
+            // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P over the S columns
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
+            uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
+            exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
             {
                 float a0, a1, b0, b1;
                 ptx::unpack2(sum2a, a0, a1);
@@ -603,18 +686,23 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(4 + 3 * jj);
         }
 
-        if (ok) ok = warp_wait(bar_o_full, 0, kDevTimeoutSoftmaxO, a.status, s_abort, lane);
+        // all tiles handed over; a slower warp of the quarter may still ask for a new reference
+        while (ok) {
+            const int r = wait_or_request(bar_o_full, 0, kDevTimeoutSoftmaxO);
+            if (r == 0) break;
+            ok = (r == 1) && move_reference(ntiles, false, 0.f);
+        }
+
         if (ok) {
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(60);
             // the row sum is the sum over the row's threads (same reference in all)
-            float* xch = s_xch + (ntiles & 1) * (kParts * 128);
+            float* xch = s_xch + kParts * 128;
             xch[part * 128 + r_tile] = l;
-            meet_arrive();
-            ok = meet_wait(ntiles);
+            ok = meet(bar_xch, 1);
         }
         if (ok) {
-            const float* xch = s_xch + (ntiles & 1) * (kParts * 128);
+            const float* xch = s_xch + kParts * 128;
             l = 0.f;
 #pragma unroll
             for (int c = 0; c < kParts; ++c) l += xch[c * 128 + r_tile];
