@@ -268,7 +268,7 @@ def run_ours(args, rank, world, local_rank, dist):
         "steps_per_s": round(aggregate_steps_per_s(us_step, world), 1),
         "step_roofline_frac": round(max(t_flop_us, t_hbm_us) / us_step, 4),
         "roofline": {
-            "kernel": "attn_tc_kernel (evlnStepAttention)", "bound": "tensor",
+            "kernel": "attn_pair_kernel (evlnStepAttention)", "bound": "tensor",
             "achieved": round(achieved_tf, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
             "frac": round(achieved_tf / peaks["bf16_tflops"], 4), "peak_kind": f"{peaks_kind} burst bf16",
             "traffic": None, "us_per_launch": round(us_attn, 3),

@@ -112,6 +112,22 @@ def test_tc_kernel_planted_high_logit_keys(handle):
     _run(handle, cfg, num_splits=3, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2)
 
 
+def test_tc_kernel_reference_moves_in_late_tiles(handle):
+    # Cached keys scaled up so far that, for about half of the rows, a score in a late KV tile
+    # exceeds the row's first-tile maximum by much more than 2^64 (twice, and once more inside the
+    # new frame): the softmax threads have to move the row's reference and rescale what they have
+    # accumulated and handed over.  Rows for which the scaled key scores negative must not move.
+    cfg = dataclasses.replace(W.STEP_7B, name="moves", cache_len=1700, num_new=96, input_scale=1.0, seed=11)
+    x = W.make_step_inputs(cfg)
+    x["k_cache"][700] *= 48.0
+    x["k_cache"][1410:1412] *= 128.0
+    x["k_new"][50] *= 250.0
+    # the winning scores are several hundred: fp32 accumulation on the tensor core resolves them to
+    # a few 1e-5 relative, which is what the log-sum-exp gate allows here
+    for splits in (1, 2):
+        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
+
+
 def test_tc_matches_simt_kernel_on_device(handle):
     cfg = dataclasses.replace(W.STEP_7B, name="cross", cache_len=700, num_new=90, seed=8)
     a, _ = _run(handle, cfg)
