@@ -506,7 +506,10 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
         const int r_local = row0 + r_tile;                 // packed row within the episode
         const bool row_valid = r_local < rows_valid;
-        const int bound = row_valid ? w.L + r_local / a.G : -1;   // last visible key index
+        // last visible key index; a padding row (beyond the episode's rows: its Q is zero fill or
+        // another episode's) is never stored, so it takes everything unmasked rather than making its
+        // warp mask every tile
+        const int bound = row_valid ? w.L + r_local / a.G : 0x3fffffff;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
         const uint32_t t_o = t_lane + kColO + part * 32;
         const uint32_t p_full0 = ptx::map_to_cta(bar_p_full, 0);
