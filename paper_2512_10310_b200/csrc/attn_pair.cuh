@@ -312,30 +312,34 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         ptx::prefetch_tensormap(&tm_q);
         ptx::prefetch_tensormap(&tm_k);
         ptx::prefetch_tensormap(&tm_v);
+        if (!PAGED) {
+            // this CTA's halves of the first K tiles and of the first V tile on their way into L2 while
+            // the pair sets up (cached rows; a row the previous kernel is still writing stays coherent)
+            const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
+            for (int jj = 0; jj < pre; ++jj) {
+                const int key0 = (w.j0 + jj) * kTileN + (int)rank * 64;
+                ptx::tma_prefetch_3d(&tm_k, 0, key0, w.g);
+                ptx::tma_prefetch_3d(&tm_k, 64, key0, w.g);
+            }
+            ptx::tma_prefetch_3d(&tm_v, 64 * (int)rank, w.j0 * kTileN, w.g);
+        }
     }
-    if (threadIdx.x == 0) {
-        ptx::mbar_init(bar_q_full, 2);
-        for (int s = 0; s < kKStages; ++s) {
-            ptx::mbar_init(bar_k_full + 8 * s, 2);
-            ptx::mbar_init(bar_k_empty + 8 * s, 1);
+    if (warp == 2 || warp == 3) {
+        // one barrier per thread: arrival counts in the order of the barrier area
+        const int i = (int)threadIdx.x - 64;
+        constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 4 + 1 + 4 + 4;
+        if (i < kNumBars) {
+            int count = 1;
+            if (i < 1 + kKStages + kVStages) count = 2;                                   // q_full, k_full, v_full
+            else if (i < 1 + 2 * kKStages + 2 * kVStages + kScoreBufs) count = 1;         // k_empty, v_empty, s_full
+            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs) count = 8 * kParts;   // p_full: 4 * kParts warps per CTA
+            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5) count = 1;  // pv_done, o_full
+            else count = kParts;                                                          // xch, rare
+            ptx::mbar_init(bar_base + 8 * i, count);
+            ptx::fence_barrier_init();
         }
-        for (int s = 0; s < kVStages; ++s) {
-            ptx::mbar_init(bar_v_full + 8 * s, 2);
-            ptx::mbar_init(bar_v_empty + 8 * s, 1);
-        }
-        for (int b = 0; b < kScoreBufs; ++b) {
-            ptx::mbar_init(bar_s_full + 8 * b, 1);
-            ptx::mbar_init(bar_p_full + 8 * b, 8 * kParts);      // 4 * kParts softmax warps in each CTA
-        }
-        ptx::mbar_init(bar_o_full, 1);
-        for (int q = 0; q < 4; ++q) {
-            ptx::mbar_init(bar_pv_done + 8 * q, 1);
-            ptx::mbar_init(bar_xch + 8 * q, kParts);
-            ptx::mbar_init(bar_rare + 8 * q, kParts);
-            s_req[q] = 0;
-        }
-        *s_abort = 0;
-        ptx::fence_barrier_init();
+        if (i < 4) s_req[i] = 0;
+        if (i == 0) *s_abort = 0;
     }
     if (warp == 1) {
         ptx::tmem_alloc_pair(tmem_slot, 512);

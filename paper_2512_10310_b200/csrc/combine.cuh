@@ -55,6 +55,25 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
     const long prow0 = (long)g * a.rows + row;
 
     float my_lse = (lane < S) ? a.lse_part[prow0 + lane * stride_s] : -INFINITY;
+    // the first partial rows do not depend on the weights: their loads go out with the lse load
+    constexpr int kPre = 4;
+    float pre[kPre][C];
+#pragma unroll
+    for (int s = 0; s < kPre; ++s) {
+        if (s < S) {
+            const float* op = a.o_part + (prow0 + s * stride_s) * D + lane * C;
+            if (C == 4) {
+                float4 x = *reinterpret_cast<const float4*>(op);
+                pre[s][0] = x.x; pre[s][1] = x.y; pre[s][2] = x.z; pre[s][3] = x.w;
+            } else {
+#pragma unroll
+                for (int c = 0; c < C; ++c) pre[s][c] = op[c];
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) pre[s][c] = 0.f;
+        }
+    }
     float M = my_lse;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
@@ -66,7 +85,13 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
     float acc[C];
 #pragma unroll
     for (int c = 0; c < C; ++c) acc[c] = 0.f;
-    for (int s = 0; s < S; ++s) {
+#pragma unroll
+    for (int s = 0; s < kPre; ++s) {
+        const float ws = __shfl_sync(0xffffffffu, w, s);      // 0 for s >= S and for empty splits
+#pragma unroll
+        for (int c = 0; c < C; ++c) acc[c] = fmaf(ws, pre[s][c], acc[c]);
+    }
+    for (int s = kPre; s < S; ++s) {
         const float ws = __shfl_sync(0xffffffffu, w, s);
         if (ws == 0.f) continue;                               // uniform across the warp
         const float* op = a.o_part + (prow0 + s * stride_s) * D + lane * C;
