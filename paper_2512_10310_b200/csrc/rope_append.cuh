@@ -64,7 +64,9 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
         const int j = threadIdx.x;
         double omega = exp2(-(2.0 * (double)j / (double)D) * a.log2_theta);
         double s, c;
-        sincos((double)pos * omega, &s, &c);
+        // sin/cos(pos * omega) through sincospi: its range reduction is exact and cheap, where a
+        // plain sincos of an argument of thousands of radians takes the slow reduction path
+        sincospi((double)pos * omega * 0.31830988618379067154, &s, &c);
         s_cos[j] = c;
         s_sin[j] = s;
     }
