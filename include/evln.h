@@ -10,7 +10,9 @@
  *
  *     evlnRopeAppend  ->  evlnStepAttention  ->  evlnStepCombine
  *
- * plus evlnPaged* variants for a batch of episodes whose caches live in a page pool.
+ * plus evlnPaged* variants for a batch of episodes whose caches live in a page pool, and
+ * evlnStoreAppend / evlnSampleFrames / evlnGatherRope for the paper's un-rotated store that a
+ * frame sampler re-indexes every step (declared at the end of this file).
  *
  * Conventions
  *  - Every data pointer is DEVICE memory owned by the caller unless its name starts with
@@ -207,6 +209,57 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t handle, const evlnPagedParams* pa
 evlnStatus_t evlnStepAttentionNoAlloc(const evlnStepParams* params, const void* q_rot,
                                       const void* k_cache, const void* v_cache, void* out,
                                       float* lse_out, void* stream);
+
+/* ---- un-rotated store + frame sampler (Sec. 3.2, "store the KV cache prior to the rotation",
+ *      frame samplers "uniform" and "sliding window") -------------------------------------
+ *
+ * The episode's raw keys and values (as projected, NOT rotated) live in a store
+ * [Hkv, store_capacity, D] per layer.  Every step the caller
+ *   1. appends the new frame's raw K/V to the store                    (evlnStoreAppend),
+ *   2. lets a sampler choose the history frames to keep                (evlnSampleFrames, host),
+ *   3. lays the kept segments out back to back in a working cache [Hkv, work_capacity, D],
+ *      the token landing in slot p rotated at position p               (evlnGatherRope),
+ *   4. runs the usual step on that working cache with cache_len = kept tokens:
+ *      evlnRopeAppend (new frame at the next contiguous positions) -> evlnStepAttention ->
+ *      evlnStepCombine.
+ */
+typedef struct {
+    size_t struct_size;      /* sizeof(evlnGatherParams)                                     */
+    int dtype;               /* evlnDType_t of store and working cache                       */
+    int num_kv_heads;        /* Hkv                                                          */
+    int head_dim;            /* D: 64 or 128                                                 */
+    int store_capacity;      /* token slots per kv head in k_store / v_store                 */
+    int work_capacity;       /* token slots per kv head in k_work / v_work                   */
+    double rope_theta;
+} evlnGatherParams;
+
+typedef enum { EVLN_SAMPLE_UNIFORM = 0, EVLN_SAMPLE_SLIDING = 1 } evlnSampler_t;
+
+/* Host helper, no GPU work.  Chooses at most `budget` of the history frames 0 .. num_frames-1
+ * and writes their indices in ascending order to h_indices (room for `budget` ints).
+ *   UNIFORM: all frames if num_frames <= budget, else frame round(k (num_frames-1)/(budget-1)),
+ *            k = 0 .. budget-1 (first and last frame always kept; `stride` ignored).
+ *   SLIDING: frames num_frames-1, num_frames-1-stride, ... (the most recent ones, `stride`
+ *            apart, stride >= 1), at most `budget` of them.
+ * Returns the number of indices written, or -1 for bad arguments.                            */
+int evlnSampleFrames(int sampler, int num_frames, int budget, int stride, int* h_indices);
+
+/* Raw (un-rotated) k_new / v_new [n, Hkv, D] (token strides in elements) -> store slots
+ * store_len .. store_len+n-1.  EVLN_CACHE_FULL if they do not fit.                           */
+evlnStatus_t evlnStoreAppend(evlnHandle_t handle, const evlnGatherParams* params, const void* k_new,
+                             const void* v_new, long k_stride_tok, long v_stride_tok, int store_len,
+                             int num_new, void* k_store, void* v_store, void* stream);
+
+/* Kept segments s = 0 .. num_segments-1 (at most 256): store slots
+ * [h_seg_src[s], h_seg_src[s] + h_seg_len[s]) go to the working cache back to back, in the
+ * order given; the key landing in working slot p is rotated by RoPE at position p, the value
+ * is copied bit-exactly.  *h_total (optional) receives the number of tokens laid out.
+ * Slots of the working cache beyond that are not touched.  EVLN_INVALID_VALUE for a segment
+ * outside the store, EVLN_CACHE_FULL if the working cache is too small.                      */
+evlnStatus_t evlnGatherRope(evlnHandle_t handle, const evlnGatherParams* params, int num_segments,
+                            const int* h_seg_src, const int* h_seg_len, const void* k_store,
+                            const void* v_store, void* k_work, void* v_work, int* h_total,
+                            void* stream);
 
 #ifdef __cplusplus
 }

@@ -16,7 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "lib", "libevln.so")
 _SOURCES = ["evln_api.cu", "attn_pair.cuh", "attn_simt.cuh", "combine.cuh", "rope_append.cuh",
-            "common.cuh", "ptx_sm100.cuh"]
+            "common.cuh", "ptx_sm100.cuh", "gather_rope.cuh"]
 
 EVLN_OK, EVLN_INVALID_VALUE, EVLN_NOT_SUPPORTED, EVLN_CACHE_FULL = 0, 1, 2, 3
 EVLN_WORKSPACE_TOO_SMALL, EVLN_CUDA_ERROR, EVLN_DEVICE_TIMEOUT = 4, 5, 6
@@ -29,6 +29,7 @@ EXPORTS = [
     "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine",
     "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
     "evlnStepAttentionNoAlloc",
+    "evlnSampleFrames", "evlnStoreAppend", "evlnGatherRope",
 ]
 EVLN_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -45,6 +46,14 @@ class evlnPagedParams(Structure):
                 ("num_kv_heads", c_int), ("head_dim", c_int), ("batch", c_int),
                 ("page_size", c_int), ("num_pages", c_int), ("max_pages_per_seq", c_int),
                 ("kv_chunk_tiles", c_int), ("softmax_scale", c_float), ("rope_theta", c_double)]
+
+
+class evlnGatherParams(Structure):
+    _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_kv_heads", c_int), ("head_dim", c_int),
+                ("store_capacity", c_int), ("work_capacity", c_int), ("rope_theta", c_double)]
+
+
+EVLN_SAMPLE_UNIFORM, EVLN_SAMPLE_SLIDING = 0, 1
 
 
 class EvlnError(RuntimeError):
@@ -106,6 +115,12 @@ def lib():
                                              c_void_p, c_size_t, c_void_p]
         L.evlnPagedStepCombine.argtypes = [c_void_p, gp, c_void_p, ip, ip, c_void_p, c_void_p, c_void_p]
         L.evlnStepAttentionNoAlloc.argtypes = [pp, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        qp = POINTER(evlnGatherParams)
+        L.evlnSampleFrames.argtypes = [c_int, c_int, c_int, c_int, POINTER(c_int)]
+        L.evlnStoreAppend.argtypes = [c_void_p, qp, c_void_p, c_void_p, c_long, c_long, c_int, c_int, c_void_p,
+                                      c_void_p, c_void_p]
+        L.evlnGatherRope.argtypes = [c_void_p, qp, c_int, POINTER(c_int), POINTER(c_int), c_void_p, c_void_p,
+                                     c_void_p, c_void_p, POINTER(c_int), c_void_p]
         for name in EXPORTS:
             if name != "evlnGetErrorString":
                 getattr(L, name).restype = c_int
@@ -265,3 +280,33 @@ def evlnStepAttentionNoAlloc(params, q_rot, k_cache, v_cache, out, lse_out=None,
     _check(lib().evlnStepAttentionNoAlloc(byref(params), _ptr(q_rot), _ptr(k_cache), _ptr(v_cache),
                                           _ptr(out), _ptr(lse_out), _stream(stream)),
            "evlnStepAttentionNoAlloc")
+
+
+def gather_params(dtype, num_kv_heads, head_dim, store_capacity, work_capacity, rope_theta) -> evlnGatherParams:
+    code = {"bf16": EVLN_BF16, "f32": EVLN_F32}.get(dtype, dtype)
+    return evlnGatherParams(ctypes.sizeof(evlnGatherParams), code, num_kv_heads, head_dim, store_capacity,
+                            work_capacity, rope_theta)
+
+
+def evlnSampleFrames(sampler: int, num_frames: int, budget: int, stride: int = 1):
+    """Host helper: indices of the history frames the sampler keeps (ascending)."""
+    buf = (c_int * max(budget, 1))()
+    cnt = lib().evlnSampleFrames(int(sampler), int(num_frames), int(budget), int(stride), buf)
+    if cnt < 0:
+        raise EvlnError(EVLN_INVALID_VALUE, "evlnSampleFrames")
+    return [int(buf[i]) for i in range(cnt)]
+
+
+def evlnStoreAppend(handle, params, k_new, v_new, store_len, k_store, v_store, stream=None):
+    _check(lib().evlnStoreAppend(handle, byref(params), _ptr(k_new), _ptr(v_new), int(k_new.stride(0)),
+                                 int(v_new.stride(0)), int(store_len), int(k_new.shape[0]), _ptr(k_store),
+                                 _ptr(v_store), _stream(stream)), "evlnStoreAppend")
+
+
+def evlnGatherRope(handle, params, seg_src, seg_len, k_store, v_store, k_work, v_work, stream=None) -> int:
+    """Lays the kept store segments out in the working cache; returns the number of tokens laid out."""
+    total = c_int(0)
+    _check(lib().evlnGatherRope(handle, byref(params), len(seg_src), _ints(seg_src), _ints(seg_len), _ptr(k_store),
+                                _ptr(v_store), _ptr(k_work), _ptr(v_work), byref(total), _stream(stream)),
+           "evlnGatherRope")
+    return int(total.value)

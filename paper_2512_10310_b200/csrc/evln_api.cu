@@ -14,6 +14,7 @@
 #include "attn_simt.cuh"
 #include "attn_pair.cuh"
 #include "combine.cuh"
+#include "gather_rope.cuh"
 #include "common.cuh"
 #include "rope_append.cuh"
 
@@ -598,6 +599,108 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t h, const evlnPagedParams* p, cons
 }
 
 }  // extern "C"
+
+// ---- un-rotated store + frame sampler ------------------------------------------------------
+
+namespace {
+evlnStatus_t check_gather_params(evlnHandle_t h, const evlnGatherParams* p)
+{
+    if (!h || !p) return EVLN_INVALID_VALUE;
+    if (p->struct_size != sizeof(evlnGatherParams)) return EVLN_INVALID_VALUE;
+    if (p->dtype != EVLN_BF16 && p->dtype != EVLN_F32) return EVLN_INVALID_VALUE;
+    if (p->num_kv_heads <= 0 || p->store_capacity < 0 || p->work_capacity < 0) return EVLN_INVALID_VALUE;
+    if (!(p->rope_theta > 0.0)) return EVLN_INVALID_VALUE;
+    if (p->head_dim != 64 && p->head_dim != 128) return EVLN_NOT_SUPPORTED;
+    return EVLN_OK;
+}
+}  // namespace
+
+extern "C" int evlnSampleFrames(int sampler, int num_frames, int budget, int stride, int* h_indices)
+{
+    if (num_frames < 0 || budget < 0 || !h_indices) return -1;
+    if (num_frames == 0 || budget == 0) return 0;
+    if (sampler == EVLN_SAMPLE_UNIFORM) {
+        if (num_frames <= budget) {
+            for (int i = 0; i < num_frames; ++i) h_indices[i] = i;
+            return num_frames;
+        }
+        if (budget == 1) { h_indices[0] = num_frames - 1; return 1; }
+        for (int k = 0; k < budget; ++k)      // round(k (N-1) / (B-1)), halves up
+            h_indices[k] = (int)((2L * k * (num_frames - 1) + (budget - 1)) / (2L * (budget - 1)));
+        return budget;
+    }
+    if (sampler == EVLN_SAMPLE_SLIDING) {
+        if (stride < 1) return -1;
+        int count = 0;
+        for (int f = num_frames - 1; f >= 0 && count < budget; f -= stride) ++count;
+        for (int k = 0; k < count; ++k) h_indices[k] = num_frames - 1 - (count - 1 - k) * stride;
+        return count;
+    }
+    return -1;
+}
+
+extern "C" evlnStatus_t evlnStoreAppend(evlnHandle_t h, const evlnGatherParams* p, const void* k_new,
+                                        const void* v_new, long k_stride_tok, long v_stride_tok, int store_len,
+                                        int num_new, void* k_store, void* v_store, void* stream)
+{
+    evlnStatus_t s = check_gather_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (store_len < 0 || num_new < 0) return EVLN_INVALID_VALUE;
+    if ((long)store_len + num_new > (long)p->store_capacity) return EVLN_CACHE_FULL;
+    if (num_new == 0) return EVLN_OK;
+    if (!k_new || !v_new || !k_store || !v_store) return EVLN_INVALID_VALUE;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_store) || !aligned16(v_store)) return EVLN_INVALID_VALUE;
+    const int vec = 16 / elem_bytes(p->dtype);
+    const long row = (long)p->num_kv_heads * p->head_dim;
+    if (k_stride_tok < row || v_stride_tok < row || k_stride_tok % vec || v_stride_tok % vec) return EVLN_INVALID_VALUE;
+    GatherArgs a = {};
+    a.k_src = k_new; a.v_src = v_new; a.k_dst = k_store; a.v_dst = v_store;
+    a.k_stride = k_stride_tok; a.v_stride = v_stride_tok;
+    a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.dst_cap = p->store_capacity; a.first_slot = store_len; a.num_tokens = num_new;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->dtype == EVLN_BF16) launch_pdl(store_append_kernel<__nv_bfloat16>, dim3(num_new), dim3(128), 0, st, a);
+    else launch_pdl(store_append_kernel<float>, dim3(num_new), dim3(128), 0, st, a);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+extern "C" evlnStatus_t evlnGatherRope(evlnHandle_t h, const evlnGatherParams* p, int num_segments,
+                                       const int* h_seg_src, const int* h_seg_len, const void* k_store,
+                                       const void* v_store, void* k_work, void* v_work, int* h_total, void* stream)
+{
+    evlnStatus_t s = check_gather_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (num_segments < 0 || (num_segments > 0 && (!h_seg_src || !h_seg_len))) return EVLN_INVALID_VALUE;
+    if (num_segments > kMaxSegments) return EVLN_NOT_SUPPORTED;
+    SegList segs;
+    memset(&segs, 0, sizeof(segs));
+    long total = 0;
+    for (int i = 0; i < num_segments; ++i) {
+        if (h_seg_src[i] < 0 || h_seg_len[i] < 0 || (long)h_seg_src[i] + h_seg_len[i] > (long)p->store_capacity)
+            return EVLN_INVALID_VALUE;
+        segs.src[i] = h_seg_src[i];
+        segs.dst_off[i] = (int)total;
+        total += h_seg_len[i];
+        if (total > (long)p->work_capacity) return EVLN_CACHE_FULL;
+    }
+    for (int i = num_segments; i <= kMaxSegments; ++i) segs.dst_off[i] = (int)total;
+    if (h_total) *h_total = (int)total;
+    if (total == 0) return EVLN_OK;
+    if (!k_store || !v_store || !k_work || !v_work) return EVLN_INVALID_VALUE;
+    if (!aligned16(k_store) || !aligned16(v_store) || !aligned16(k_work) || !aligned16(v_work)) return EVLN_INVALID_VALUE;
+    GatherArgs a = {};
+    a.k_src = k_store; a.v_src = v_store; a.k_dst = k_work; a.v_dst = v_work;
+    a.Hkv = p->num_kv_heads; a.D = p->head_dim;
+    a.src_cap = p->store_capacity; a.dst_cap = p->work_capacity;
+    a.num_tokens = (int)total; a.num_segments = num_segments;
+    a.log2_theta = log2(p->rope_theta);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (p->dtype == EVLN_BF16) launch_pdl(gather_rope_kernel<__nv_bfloat16>, dim3((int)total), dim3(128), 0, st, a, segs);
+    else launch_pdl(gather_rope_kernel<float>, dim3((int)total), dim3(128), 0, st, a, segs);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
 
 // ---- allocation-free variant --------------------------------------------------------------
 

@@ -35,6 +35,7 @@ def test_struct_sizes_match_the_header_layout():
     # 9 ints + float + double after a size_t: no hidden padding surprises on LP64
     assert ctypes.sizeof(B.evlnStepParams) == 56
     assert ctypes.sizeof(B.evlnPagedParams) == 56
+    assert ctypes.sizeof(B.evlnGatherParams) == 40
 
 
 def test_error_strings(lib):
