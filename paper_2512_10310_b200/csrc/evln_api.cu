@@ -124,7 +124,9 @@ int choose_splits_tc(int units_total, int nkv_max, int nkv_min, int num_sms)
     const int smax = nkv_min < kMaxSplits ? (nkv_min < 1 ? 1 : nkv_min) : kMaxSplits;
     for (int s = 1; s <= smax; ++s) {
         const double waves = ceil((double)units_total * s / pairs);
-        const double cost = waves * (ceil((double)nkv_max / s) + 2.0) + 0.3 * s;
+        // per work item: set-up, first-tile latency, partial write-out and teardown cost about as
+        // much as 7 KV tiles (measured); every split adds about half a tile of combine work
+        const double cost = waves * (ceil((double)nkv_max / s) + 7.0) + 0.5 * s;
         if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
     }
     return best;

@@ -70,10 +70,11 @@ def test_no_alloc_rejects_oversized_problems():
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
     torch.cuda.set_device(0)
-    # 70B-class long-history shape: its split workspace is far beyond the built-in scratch
+    # 70B-class long-history shape with 8 KV splits asked for: 67 MB of split partials, far beyond
+    # the built-in scratch (the check comes before any launch, so the dummy buffers are never used)
     cfg = W.LONG_70B
     p = B.step_params("bf16", cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.cache_len, cfg.num_new,
-                      cfg.cache_len + cfg.num_new, cfg.rope_theta)
+                      cfg.cache_len + cfg.num_new, cfg.rope_theta, num_splits=8)
     buf = torch.zeros(4096, dtype=torch.uint8, device="cuda:0")
     with pytest.raises(B.EvlnError) as e:
         B.evlnStepAttentionNoAlloc(p, buf, buf, buf, buf, None)
