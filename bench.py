@@ -114,7 +114,7 @@ def physical_gpu_index(local_index: int) -> int:
 class LayerRing:
     """Device buffers of RING_LAYERS independent layers of the workload + pinned host copies."""
 
-    def __init__(self, B, handle, cfg, dev, layers):
+    def __init__(self, B, handle, cfg, dev, layers, random_device_inputs=False):
         self.B, self.h, self.cfg, self.dev = B, handle, cfg, dev
         L, n, Hq, Hkv, D = cfg.cache_len, cfg.num_new, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
         self.p = B.step_params(cfg.dtype, Hq, Hkv, D, L, n, L + n, cfg.rope_theta)
@@ -124,6 +124,17 @@ class LayerRing:
         self.layers = []
         dt = cfg.torch_dtype
         for l in range(layers):
+            if random_device_inputs:
+                # same distribution, drawn on the device (the cache-length sweep needs no host copies)
+                gen = torch.Generator(device=dev).manual_seed(cfg.seed * 7919 + l)
+                mk = lambda *sh: (torch.randn(*sh, generator=gen, device=dev, dtype=torch.float32) * cfg.input_scale).to(dt)
+                self.layers.append(dict(
+                    kc=mk(Hkv, L + n, D), vc=mk(Hkv, L + n, D), q=mk(n, Hq, D), k=mk(n, Hkv, D), v=mk(n, Hkv, D),
+                    q_rot=torch.empty(qbytes, dtype=torch.uint8, device=dev),
+                    ws=torch.empty(wbytes, dtype=torch.uint8, device=dev),
+                    out=torch.empty((n, Hq, D), dtype=dt, device=dev)))
+                kc = self.layers[-1]["kc"]
+                continue
             x = W.make_step_inputs(dataclasses.replace(cfg, seed=cfg.seed * 7919 + l))
             kc = torch.zeros((Hkv, L + n, D), dtype=dt, device=dev)
             vc = torch.zeros((Hkv, L + n, D), dtype=dt, device=dev)
@@ -237,6 +248,35 @@ def run_ours(args, rank, world, local_rank, dist):
     us_step = max_over_ranks(ms * 1e3 / steps)
     us_attn = max_over_ranks(ms_attn * 1e3 / steps)
     us_e2e = max_over_ranks(ms_e2e * 1e3 / e2e_steps)
+
+    # The metric is quoted against the cache length: the same layer-step at other L (7B-class shape),
+    # a short measurement each, on rank 0 of a single-GPU run only.
+    h2d = sum(t.numel() * t.element_size() for t in ring.layers[0]["host_in"])
+    d2h = ring.layers[0]["host_out"].numel() * ring.layers[0]["host_out"].element_size()
+    by_len = []
+    if world == 1 and not args.no_sweep:
+        del g_step, g_attn
+        ring.layers.clear()
+        torch.cuda.empty_cache()
+        peaks_s, _ = load_peaks()
+        for L in (1024, 8192, 16384, 32768):
+            c = dataclasses.replace(cfg, name=f"step_7b_L{L}", cache_len=L)
+            kv_bytes = 2 * (L + c.num_new) * c.num_kv_heads * c.head_dim * 2
+            layers = max(2, min(RING_LAYERS, int(2.2 * L2_BYTES / kv_bytes) + 1))
+            r = LayerRing(B, handle, c, dev, layers, random_device_inputs=True)
+            gs, ga = capture(r.step, layers), capture(r.attention_only, layers)
+            reps = max(3, 640 // layers)
+            for _ in range(3):
+                gs.replay()
+            t_s = timed(gs.replay, reps, barrier) * 1e3 / (reps * layers)
+            t_a = timed(ga.replay, reps, barrier) * 1e3 / (reps * layers)
+            roof = max(c.flops() / (peaks_s["bf16_tflops"] * 1e12), c.algorithmic_bytes() / (peaks_s["hbm_gbs"] * 1e9)) * 1e6
+            by_len.append({"cache_len": L, "us_per_step": round(t_s, 2), "attention_us": round(t_a, 2),
+                           "attention_tflops": round(c.flops() / t_a / 1e6, 1), "kv_splits": r.splits,
+                           "step_roofline_frac": round(roof / t_s, 4)})
+            del gs, ga, r
+            torch.cuda.empty_cache()
+        assert B.evlnGetDeviceStatus(handle) == 0, "a kernel gave up on a bounded wait"
     B.evlnDestroy(handle)
     if rank != 0:
         return None
@@ -247,8 +287,6 @@ def run_ours(args, rank, world, local_rank, dist):
     t_flop_us = flops / (peaks["bf16_tflops"] * 1e12) * 1e6
     t_hbm_us = abytes / (peaks["hbm_gbs"] * 1e9) * 1e6
     achieved_tf = flops / (us_attn * 1e-6) / 1e12
-    h2d = sum(t.numel() * t.element_size() for t in ring.layers[0]["host_in"])
-    d2h = ring.layers[0]["host_out"].numel() * ring.layers[0]["host_out"].element_size()
     line = {
         "metric": "new-frame step-attention latency", "value": round(us_step, 3), "unit": "us/step",
         "n_gpus": world, "steps": steps, "warmup": warm, "ms_per_step": us_step / 1e3,
@@ -280,6 +318,8 @@ def run_ours(args, rank, world, local_rank, dist):
         "gpu_launches": 3 * steps,
         "clocks": clocks,
     }
+    if by_len:
+        line["by_cache_len"] = by_len
     return line
 
 
@@ -369,6 +409,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short cache-length sweep")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
