@@ -261,6 +261,23 @@ evlnStatus_t evlnGatherRope(evlnHandle_t handle, const evlnGatherParams* params,
                             const void* v_store, void* k_work, void* v_work, int* h_total,
                             void* stream);
 
+/* ---- host-resident store (Sec. 3.2, "Memory Management": the cache is offloaded to the CPU and
+ *      only the segments the sampler selects are reloaded) ------------------------------------
+ *
+ * The full raw store of an episode may live in PINNED host memory, [Hkv, host_capacity, D],
+ * while the device store only has room for the segments in use.  evlnStoreOffload copies token
+ * slots of the device store to the host store, evlnStoreFetch copies token slots of the host
+ * store into the device store; each is one strided DMA per tensor (all kv heads at once),
+ * enqueued on `stream`, no kernel.  Which frames are resident, and where, is the caller's
+ * bookkeeping (paper_2512_10310_b200/residency.py has one).  h_k_store / h_v_store must be
+ * page-locked for the copies to be asynchronous.                                               */
+evlnStatus_t evlnStoreOffload(evlnHandle_t handle, const evlnGatherParams* params, const void* k_store,
+                              const void* v_store, int src_slot, int len, void* h_k_store, void* h_v_store,
+                              int host_capacity, int dst_slot, void* stream);
+evlnStatus_t evlnStoreFetch(evlnHandle_t handle, const evlnGatherParams* params, const void* h_k_store,
+                            const void* h_v_store, int host_capacity, int src_slot, int len, void* k_store,
+                            void* v_store, int dst_slot, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

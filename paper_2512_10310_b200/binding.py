@@ -29,7 +29,7 @@ EXPORTS = [
     "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine",
     "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
     "evlnStepAttentionNoAlloc",
-    "evlnSampleFrames", "evlnStoreAppend", "evlnGatherRope",
+    "evlnSampleFrames", "evlnStoreAppend", "evlnGatherRope", "evlnStoreOffload", "evlnStoreFetch",
 ]
 EVLN_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -121,6 +121,10 @@ def lib():
                                       c_void_p, c_void_p]
         L.evlnGatherRope.argtypes = [c_void_p, qp, c_int, POINTER(c_int), POINTER(c_int), c_void_p, c_void_p,
                                      c_void_p, c_void_p, POINTER(c_int), c_void_p]
+        L.evlnStoreOffload.argtypes = [c_void_p, qp, c_void_p, c_void_p, c_int, c_int, c_void_p, c_void_p, c_int, c_int,
+                                       c_void_p]
+        L.evlnStoreFetch.argtypes = [c_void_p, qp, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_int,
+                                     c_void_p]
         for name in EXPORTS:
             if name != "evlnGetErrorString":
                 getattr(L, name).restype = c_int
@@ -310,3 +314,17 @@ def evlnGatherRope(handle, params, seg_src, seg_len, k_store, v_store, k_work, v
                                 _ptr(v_store), _ptr(k_work), _ptr(v_work), byref(total), _stream(stream)),
            "evlnGatherRope")
     return int(total.value)
+
+
+def evlnStoreOffload(handle, params, k_store, v_store, src_slot, length, h_k_store, h_v_store, dst_slot, stream=None):
+    """Device store slots -> pinned host store ``[Hkv, host_capacity, D]`` (asynchronous DMA)."""
+    _check(lib().evlnStoreOffload(handle, byref(params), _ptr(k_store), _ptr(v_store), int(src_slot), int(length),
+                                  _ptr(h_k_store), _ptr(h_v_store), int(h_k_store.shape[1]), int(dst_slot),
+                                  _stream(stream)), "evlnStoreOffload")
+
+
+def evlnStoreFetch(handle, params, h_k_store, h_v_store, src_slot, length, k_store, v_store, dst_slot, stream=None):
+    """Pinned host store slots -> device store slots (asynchronous DMA)."""
+    _check(lib().evlnStoreFetch(handle, byref(params), _ptr(h_k_store), _ptr(h_v_store), int(h_k_store.shape[1]),
+                                int(src_slot), int(length), _ptr(k_store), _ptr(v_store), int(dst_slot),
+                                _stream(stream)), "evlnStoreFetch")

@@ -704,6 +704,49 @@ extern "C" evlnStatus_t evlnGatherRope(evlnHandle_t h, const evlnGatherParams* p
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
 
+// ---- host-resident store: strided DMA between the pinned host store and the device store ----
+
+namespace {
+evlnStatus_t store_copy(evlnHandle_t h, const evlnGatherParams* p, const void* k_src, const void* v_src, int src_cap,
+                        int src_slot, int len, void* k_dst, void* v_dst, int dst_cap, int dst_slot, cudaStream_t st,
+                        cudaMemcpyKind kind)
+{
+    evlnStatus_t s = check_gather_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (src_slot < 0 || dst_slot < 0 || len < 0 || src_cap < 0 || dst_cap < 0) return EVLN_INVALID_VALUE;
+    if ((long)src_slot + len > (long)src_cap) return EVLN_INVALID_VALUE;
+    if ((long)dst_slot + len > (long)dst_cap) return EVLN_CACHE_FULL;
+    if (len == 0) return EVLN_OK;
+    if (!k_src || !v_src || !k_dst || !v_dst) return EVLN_INVALID_VALUE;
+    const size_t row = (size_t)p->head_dim * elem_bytes(p->dtype);       // one token of one head
+    const size_t width = row * len;
+    cudaError_t e = cudaMemcpy2DAsync((char*)k_dst + row * dst_slot, row * dst_cap, (const char*)k_src + row * src_slot,
+                                      row * src_cap, width, p->num_kv_heads, kind, st);
+    if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync((char*)v_dst + row * dst_slot, row * dst_cap, (const char*)v_src + row * src_slot,
+                              row * src_cap, width, p->num_kv_heads, kind, st);
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+}  // namespace
+
+extern "C" evlnStatus_t evlnStoreOffload(evlnHandle_t h, const evlnGatherParams* p, const void* k_store,
+                                         const void* v_store, int src_slot, int len, void* h_k_store, void* h_v_store,
+                                         int host_capacity, int dst_slot, void* stream)
+{
+    if (!p) return EVLN_INVALID_VALUE;
+    return store_copy(h, p, k_store, v_store, p->store_capacity, src_slot, len, h_k_store, h_v_store, host_capacity,
+                      dst_slot, (cudaStream_t)stream, cudaMemcpyDeviceToHost);
+}
+
+extern "C" evlnStatus_t evlnStoreFetch(evlnHandle_t h, const evlnGatherParams* p, const void* h_k_store,
+                                       const void* h_v_store, int host_capacity, int src_slot, int len, void* k_store,
+                                       void* v_store, int dst_slot, void* stream)
+{
+    if (!p) return EVLN_INVALID_VALUE;
+    return store_copy(h, p, h_k_store, h_v_store, host_capacity, src_slot, len, k_store, v_store, p->store_capacity,
+                      dst_slot, (cudaStream_t)stream, cudaMemcpyHostToDevice);
+}
+
 // ---- allocation-free variant --------------------------------------------------------------
 
 // Scratch for the split partials of evlnStepAttentionNoAlloc, part of the library image: every
