@@ -8,7 +8,7 @@
  * to the reused cache, and the n new queries attend causally to all L+n cached tokens
  * (grouped-query attention).  Per transformer layer this is three calls:
  *
- *     evlnRopeAppend  ->  evlnStepAttention  ->  evlnStepCombine
+ *     evlnRopeAppend  ->  evlnStepAttention  ->  evlnStepCombine      (or evlnStep: all three)
  *
  * plus evlnPaged* variants for a batch of episodes whose caches live in a page pool, and
  * evlnStoreAppend / evlnSampleFrames / evlnGatherRope for the paper's un-rotated store that a
@@ -138,7 +138,11 @@ evlnStatus_t evlnRopeAppend(evlnHandle_t handle, const evlnStepParams* params,
 /* Step 2 (Sec. 3.2: prefill of the current frame only, against the reused cache).
  * Causal attention of the n rotated queries over cache slots 0 .. L+n-1 (query i sees slots
  * 0 .. L+i), split over the keys; writes per-split normalised outputs and log-sum-exps into
- * `workspace`.  Must run after evlnRopeAppend of the same step on the same stream.          */
+ * `workspace`.  Must run after evlnRopeAppend of the same step on the same stream.
+ * bf16 with head_dim 128 runs on the tensor cores: CTA pairs over 256-row units of the packed
+ * query rows, or, when all n * G rows of a kv head fit one 128-row tile (the few action tokens
+ * decoded after a frame, Sec. 3.1), one CTA per (kv head, KV split) with the KV range spread
+ * over all SMs.                                                                              */
 evlnStatus_t evlnStepAttention(evlnHandle_t handle, const evlnStepParams* params,
                                const void* q_rot, const void* k_cache, const void* v_cache,
                                void* workspace, size_t workspace_bytes, void* stream);
@@ -147,6 +151,15 @@ evlnStatus_t evlnStepAttention(evlnHandle_t handle, const evlnStepParams* params
  * rounds once to the storage dtype and scatters rows back to [n, Hq, D].  lse_out may be NULL. */
 evlnStatus_t evlnStepCombine(evlnHandle_t handle, const evlnStepParams* params,
                              const void* workspace, void* out, float* lse_out, void* stream);
+
+/* The whole step in one call (Sec. 3.2): evlnRopeAppend, evlnStepAttention and evlnStepCombine
+ * with the same arguments, enqueued back to back on `stream`; same results bit for bit.
+ * All arguments are validated before the first launch; errors as for the three calls.          */
+evlnStatus_t evlnStep(evlnHandle_t handle, const evlnStepParams* params,
+                      const void* q_new, const void* k_new, const void* v_new,
+                      long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                      void* q_rot, void* k_cache, void* v_cache,
+                      void* workspace, size_t workspace_bytes, void* out, float* lse_out, void* stream);
 
 /* ---- paged cache, batch of episodes ----------------------------------------------------- */
 

@@ -26,7 +26,7 @@ EVLN_KERNEL_AUTO, EVLN_KERNEL_SIMT = 0, 1
 EXPORTS = [
     "evlnCreate", "evlnDestroy", "evlnGetErrorString", "evlnGetLastCudaError", "evlnGetDeviceStatus",
     "evlnStepNumSplits", "evlnStepWorkspaceSize", "evlnStepQRotSize",
-    "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine",
+    "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine", "evlnStep",
     "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
     "evlnStepAttentionNoAlloc",
     "evlnSampleFrames", "evlnStoreAppend", "evlnGatherRope", "evlnStoreOffload", "evlnStoreFetch",
@@ -103,6 +103,8 @@ def lib():
         L.evlnStepQRotSize.argtypes = [c_void_p, pp, POINTER(c_size_t)]
         L.evlnRopeAppend.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_long, c_long, c_long,
                                      c_void_p, c_void_p, c_void_p, c_void_p]
+        L.evlnStep.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_long, c_long, c_long, c_void_p,
+                               c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p]
         L.evlnStepAttention.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                                         c_void_p]
         L.evlnStepCombine.argtypes = [c_void_p, pp, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -243,6 +245,19 @@ def evlnStepAttention(handle, params, q_rot, k_cache, v_cache, workspace, worksp
 def evlnStepCombine(handle, params, workspace, out, lse_out=None, stream=None):
     _check(lib().evlnStepCombine(handle, byref(params), _ptr(workspace), _ptr(out), _ptr(lse_out),
                                  _stream(stream)), "evlnStepCombine")
+
+
+def evlnStep(handle, params, q_new, k_new, v_new, q_rot, k_cache, v_cache, workspace, out, lse_out=None,
+             workspace_bytes=None, stream=None, strides=None):
+    """The three calls of a step in one."""
+    if strides is None:
+        strides = (q_new.stride(0), k_new.stride(0), v_new.stride(0))
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().evlnStep(handle, byref(params), _ptr(q_new), _ptr(k_new), _ptr(v_new), int(strides[0]),
+                          int(strides[1]), int(strides[2]), _ptr(q_rot), _ptr(k_cache), _ptr(v_cache),
+                          _ptr(workspace), int(workspace_bytes), _ptr(out), _ptr(lse_out), _stream(stream)),
+           "evlnStep")
 
 
 def evlnPagedWorkspaceSize(handle, params, cache_lens, new_offsets) -> int:

@@ -52,19 +52,32 @@ namespace evln {
 
 constexpr int kTcThreads = 640;
 constexpr int kParts = 4;                             // threads per score row (32 columns each)
-constexpr int kKStages = 5, kVStages = 5;
 constexpr int kTileBytes = kTileM * 128 * 2;          // Q tile: 128 rows x 128 channels x bf16
 constexpr int kHalfBytes = kTileBytes / 2;            // 16 KB: a 64-channel half of Q; a K or V half tile
-constexpr int kSmemQOff = 0;
-constexpr int kSmemKOff = kTileBytes;
-constexpr int kSmemVOff = kSmemKOff + kKStages * kHalfBytes;
-constexpr int kSmemBarOff = kSmemVOff + kVStages * kHalfBytes;
 constexpr int kSmemBarBytes = 384;
-constexpr int kSmemXchOff = kSmemBarOff + kSmemBarBytes;          // float [2 meetings][kParts][128 rows]
-constexpr int kSmemCandOff = kSmemXchOff + 2 * kParts * 128 * 4;  // float [kParts][128 rows]: reference requests
-constexpr int kSmemReqOff = kSmemCandOff + kParts * 128 * 4;      // int [4] request flags, int [4][kParts] released tiles
 constexpr int kSmemXchBytes = 2 * kParts * 128 * 4 + kParts * 128 * 4 + 128;
-constexpr int kTcSmemBytes = kSmemXchOff + kSmemXchBytes + 1024;  // + slack to align to 1024
+
+// Shared-memory plan of a CTA.  CTAS = 2: the CTA of a pair stages half tiles (16 KB) through two
+// 5-deep rings.  CTAS = 1: a CTA on its own stages whole K / V tiles (32 KB: two 64-channel blocks
+// of 128 keys) through a 3-deep K ring and a 2-deep V ring.
+template <int CTAS>
+struct SmemPlan {
+    static constexpr int kKStages = CTAS == 2 ? 5 : 3;
+    static constexpr int kVStages = CTAS == 2 ? 5 : 2;
+    static constexpr int kStageBytes = CTAS == 2 ? kHalfBytes : kTileBytes;
+    static constexpr int kQOff = 0;
+    static constexpr int kKOff = kTileBytes;
+    static constexpr int kVOff = kKOff + kKStages * kStageBytes;
+    static constexpr int kBarOff = kVOff + kVStages * kStageBytes;
+    static constexpr int kXchOff = kBarOff + kSmemBarBytes;          // float [2 meetings][kParts][128 rows]
+    static constexpr int kCandOff = kXchOff + 2 * kParts * 128 * 4;  // float [kParts][128 rows]: reference requests
+    static constexpr int kReqOff = kCandOff + kParts * 128 * 4;      // int [4] request flags, int [4][kParts] released tiles
+    static constexpr int kBytes = kXchOff + kSmemXchBytes + 1024;    // + slack to align to 1024
+    static_assert(kKStages * kStageBytes >= 16 * 32 * 144, "the epilogue stages its rows in the K ring");
+    static_assert(kBytes <= 227 * 1024, "shared memory per CTA");
+};
+constexpr int kTcSmemBytes = SmemPlan<2>::kBytes;
+constexpr int kSoloSmemBytes = SmemPlan<1>::kBytes;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at boost clocks
 constexpr int kScoreBufs = 3;
 constexpr uint32_t kColO = 384;
@@ -194,7 +207,7 @@ struct WorkItem {
     int j0, j1;               // KV tile range
 };
 
-template <bool PAGED, typename LensT>
+template <bool PAGED, typename LensT, int UNIT_ROWS>
 __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT& lens, int item)
 {
     WorkItem w;
@@ -206,7 +219,7 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
         w.L = a.cache_len;
         w.n = a.num_new;
         w.row_base = 0;
-        const int nkv = unit_kv_tiles(w.L, w.n, a.G, w.unit, kUnitRows);
+        const int nkv = unit_kv_tiles(w.L, w.n, a.G, w.unit, UNIT_ROWS);
         w.j0 = (int)((long)w.slot * nkv / a.num_splits);
         w.j1 = (int)((long)(w.slot + 1) * nkv / a.num_splits);
     } else {
@@ -214,10 +227,10 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
         int b = 0;
         for (; b < a.batch; ++b) {
             const int n_b = lens.new_off[b + 1] - lens.new_off[b];
-            const int units = ceil_div(n_b * a.G, kUnitRows);
+            const int units = ceil_div(n_b * a.G, UNIT_ROWS);
             int per_head = 0;
             for (int u = 0; u < units; ++u)
-                per_head += ceil_div(unit_kv_tiles(lens.cache_len[b], n_b, a.G, u, kUnitRows), a.chunk_tiles);
+                per_head += ceil_div(unit_kv_tiles(lens.cache_len[b], n_b, a.G, u, UNIT_ROWS), a.chunk_tiles);
             if (rem < per_head * a.Hkv) {
                 w.b = b;
                 w.L = lens.cache_len[b];
@@ -226,7 +239,7 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
                 w.g = rem / per_head;
                 rem -= w.g * per_head;
                 for (int u = 0; u < units; ++u) {
-                    const int nkv = unit_kv_tiles(w.L, n_b, a.G, u, kUnitRows);
+                    const int nkv = unit_kv_tiles(w.L, n_b, a.G, u, UNIT_ROWS);
                     const int S = ceil_div(nkv, a.chunk_tiles);
                     if (rem < S) {
                         w.unit = u;
@@ -247,14 +260,20 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
 }
 
 // --- the kernel ---------------------------------------------------------------------------
-// Launched with a cluster of 2 CTAs along x: work item = blockIdx.x / 2, query tile = rank.
+// CTAS = 2: launched with a cluster of 2 CTAs along x: work item = blockIdx.x / 2, query tile = rank.
+// CTAS = 1: no cluster; work item = blockIdx.x, one query tile (all the rows of a kv head fit in it).
 
-template <bool PAGED, typename LensT>
-__global__ void __launch_bounds__(kTcThreads, 1)
-attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                 const __grid_constant__ CUtensorMap tm_v, const TcAttnArgs a,
-                 const __grid_constant__ LensT lens)
+template <bool PAGED, typename LensT, int CTAS>
+__device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                             const TcAttnArgs& a, const LensT& lens)
 {
+    static_assert(CTAS == 2 || !PAGED, "the paged kernel runs on CTA pairs");
+    using Plan = SmemPlan<CTAS>;
+    constexpr int kKStages = Plan::kKStages, kVStages = Plan::kVStages, kStageBytes = Plan::kStageBytes;
+    constexpr int kSmemQOff = Plan::kQOff, kSmemKOff = Plan::kKOff, kSmemVOff = Plan::kVOff;
+    constexpr int kSmemBarOff = Plan::kBarOff, kSmemXchOff = Plan::kXchOff, kSmemCandOff = Plan::kCandOff;
+    constexpr int kSmemReqOff = Plan::kReqOff;
+    constexpr int kItemRows = CTAS * kTileM;           // query rows of a work item
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -282,15 +301,22 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff) + 4;    // [4][kParts]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = ptx::cluster_ctarank();      // 0: issues the MMAs, owns the "(CTA 0)" barriers
+    const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;   // 0: issues the MMAs, owns the "(CTA 0)" barriers
     if (threadIdx.x == 0) EVLN_STAMP(0);
 
-    const WorkItem w = decode_work<PAGED, LensT>(a, lens, blockIdx.x >> 1);
+    const WorkItem w = decode_work<PAGED, LensT, kItemRows>(a, lens, CTAS == 2 ? blockIdx.x >> 1 : blockIdx.x);
     if (PAGED && w.b < 0) return;                      // both CTAs of the pair decode the same item
 
     const int rows_valid = w.n * a.G;                            // packed rows of this episode
-    const int row0 = w.unit * kUnitRows + (int)rank * kTileM;    // first row of this CTA's tile (episode-local)
+    const int row0 = w.unit * kItemRows + (int)rank * kTileM;    // first row of this CTA's tile (episode-local)
     const int ntiles = w.j1 - w.j0;
+    // Lane quarters (32 rows each) of the tile that hold rows of the episode.  A CTA on its own lets
+    // the softmax warps of the others sit out; a pair keeps all of them (both CTAs count alike).
+    int quarters = 4;
+    if (CTAS == 1) {
+        quarters = (rows_valid - row0 + 31) >> 5;
+        quarters = quarters < 1 ? 1 : (quarters > 4 ? 4 : quarters);
+    }
 
     // A split with no KV tiles (more splits than tiles): its partials are "empty".
     if (ntiles <= 0) {
@@ -322,6 +348,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 ptx::tma_prefetch_3d(&tm_k, 64, key0, w.g);
             }
             ptx::tma_prefetch_3d(&tm_v, 64 * (int)rank, w.j0 * kTileN, w.g);
+            if (CTAS == 1) ptx::tma_prefetch_3d(&tm_v, 64, w.j0 * kTileN, w.g);
         }
     }
     if (warp == 2 || warp == 3) {
@@ -330,9 +357,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 4 + 1 + 4 + 4;
         if (i < kNumBars) {
             int count = 1;
-            if (i < 1 + kKStages + kVStages) count = 2;                                   // q_full, k_full, v_full
+            if (i < 1 + kKStages + kVStages) count = CTAS;                                // q_full, k_full, v_full
             else if (i < 1 + 2 * kKStages + 2 * kVStages + kScoreBufs) count = 1;         // k_empty, v_empty, s_full
-            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs) count = 8 * kParts;   // p_full: 4 * kParts warps per CTA
+            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs) count = CTAS * quarters * kParts;   // p_full: every softmax warp
             else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5) count = 1;  // pv_done, o_full
             else count = kParts;                                                          // xch, rare
             ptx::mbar_init(bar_base + 8 * i, count);
@@ -342,13 +369,20 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (i == 0) *s_abort = 0;
     }
     if (warp == 1) {
-        ptx::tmem_alloc_pair(tmem_slot, 512);
-        ptx::tmem_relinquish_pair();
+        if (CTAS == 2) {
+            ptx::tmem_alloc_pair(tmem_slot, 512);
+            ptx::tmem_relinquish_pair();
+        } else {
+            ptx::tmem_alloc(tmem_slot, 512);
+            ptx::tmem_relinquish();
+        }
     }
     ptx::fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive();      // the other CTA's barriers exist before anything arrives on them
-    ptx::cluster_wait();
+    if (CTAS == 2) {
+        ptx::cluster_arrive();  // the other CTA's barriers exist before anything arrives on them
+        ptx::cluster_wait();
+    }
     ptx::fence_after_sync();
     const uint32_t tmem = *s_tmem;
     ptx::grid_launch_dependents();
@@ -360,29 +394,37 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             // everything this CTA reads or writes in global memory follows this thread's loads, so
             // one wait here orders the whole CTA after the kernels it depends on
             ptx::grid_dependency_wait();
-            const uint32_t q_full0 = ptx::map_to_cta(bar_q_full, 0);
+            auto expect = [&](uint32_t bar, uint32_t bytes) {
+                if (CTAS == 2) ptx::mbar_expect_tx_cluster(bar, bytes); else ptx::mbar_expect_tx(bar, bytes);
+            };
+            auto tma3 = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+                if (CTAS == 2) ptx::tma_load_3d_pair(dst, map, bar, x, y, z); else ptx::tma_load_3d(dst, map, bar, x, y, z);
+            };
+            auto on_cta0 = [&](uint32_t bar) -> uint32_t { return CTAS == 2 ? ptx::map_to_cta(bar, 0) : bar; };
             {
+                const uint32_t q_full0 = on_cta0(bar_q_full);
                 const uint32_t dst = smem_base + kSmemQOff;
                 const int qrow = w.row_base + row0;
-                ptx::mbar_expect_tx_cluster(q_full0, kTileBytes);
-                ptx::tma_load_3d_pair(dst, &tm_q, q_full0, 0, qrow, w.g);
-                ptx::tma_load_3d_pair(dst + kHalfBytes, &tm_q, q_full0, 64, qrow, w.g);
+                expect(q_full0, kTileBytes);
+                tma3(dst, &tm_q, q_full0, 0, qrow, w.g);
+                tma3(dst + kHalfBytes, &tm_q, q_full0, 64, qrow, w.g);
             }
             bool ok = true;
-            // this CTA's half of K tile j: keys [128 j + 64 rank, +64), all channels (two 64-channel blocks)
+            // K tile j.  Pair: this CTA's half, keys [128 j + 64 rank, +64), all channels (two 64-channel
+            // blocks of 64 keys).  Alone: the whole tile (two 64-channel blocks of 128 keys).
             auto load_k = [&](int jj) {
                 const int stage = jj % kKStages;
                 if (jj >= kKStages)
                     ok = wait_bounded(bar_k_empty + 8 * stage, ((jj / kKStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
                 if (!ok) return;
-                const uint32_t dst = smem_base + kSmemKOff + stage * kHalfBytes;
-                const uint32_t bar = ptx::map_to_cta(bar_k_full + 8 * stage, 0);
+                const uint32_t dst = smem_base + kSmemKOff + stage * kStageBytes;
+                const uint32_t bar = on_cta0(bar_k_full + 8 * stage);
                 const int j = w.j0 + jj;
-                ptx::mbar_expect_tx_cluster(bar, kHalfBytes);
+                expect(bar, kStageBytes);
                 if (!PAGED) {
                     const int key0 = j * kTileN + (int)rank * 64;
-                    ptx::tma_load_3d_pair(dst, &tm_k, bar, 0, key0, w.g);
-                    ptx::tma_load_3d_pair(dst + 8192, &tm_k, bar, 64, key0, w.g);
+                    tma3(dst, &tm_k, bar, 0, key0, w.g);
+                    tma3(dst + kStageBytes / 2, &tm_k, bar, 64, key0, w.g);
                 } else {
                     // a 64-token page is exactly this CTA's half; past the episode's last page the
                     // last page is read again (masked, but finite)
@@ -394,18 +436,19 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     ptx::tma_load_4d_pair(dst + 8192, &tm_k, bar, 64, 0, w.g, pg);
                 }
             };
-            // this CTA's half of V tile j: all 128 keys, channels [64 rank, +64)
+            // V tile j, all 128 keys.  Pair: channels [64 rank, +64).  Alone: both 64-channel blocks.
             auto load_v = [&](int jj) {
                 const int stage = jj % kVStages;
                 if (jj >= kVStages)
                     ok = wait_bounded(bar_v_empty + 8 * stage, ((jj / kVStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
                 if (!ok) return;
-                const uint32_t dst = smem_base + kSmemVOff + stage * kHalfBytes;
-                const uint32_t bar = ptx::map_to_cta(bar_v_full + 8 * stage, 0);
+                const uint32_t dst = smem_base + kSmemVOff + stage * kStageBytes;
+                const uint32_t bar = on_cta0(bar_v_full + 8 * stage);
                 const int j = w.j0 + jj;
-                ptx::mbar_expect_tx_cluster(bar, kHalfBytes);
+                expect(bar, kStageBytes);
                 if (!PAGED) {
-                    ptx::tma_load_3d_pair(dst, &tm_v, bar, 64 * (int)rank, j * kTileN, w.g);
+                    tma3(dst, &tm_v, bar, 64 * (int)rank, j * kTileN, w.g);
+                    if (CTAS == 1) tma3(dst + kHalfBytes, &tm_v, bar, 64, j * kTileN, w.g);
                 } else {
                     const int npages = (w.L + w.n + 63) >> 6;
                     const int p0 = 2 * j;
@@ -431,44 +474,52 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         __syncwarp();
     } else if (warp == 1 && rank == 0) {
         // ================= MMA issuer (CTA 0 of the pair) =================
-        const uint32_t idesc_s = make_idesc(false, 2 * kTileM, kTileN);
-        const uint32_t idesc_pv = make_idesc(true, 2 * kTileM, 128);
-        const uint16_t both = 3;
+        const uint32_t idesc_s = make_idesc(false, CTAS * kTileM, kTileN);
+        const uint32_t idesc_pv = make_idesc(true, CTAS * kTileM, 128);
+        auto mma_ss = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t idesc, bool acc) {
+            if (CTAS == 2) ptx::mma_ss_pair(d, ad, bd, idesc, acc); else ptx::mma_ss(d, ad, bd, idesc, acc);
+        };
+        auto mma_ts = [&](uint32_t d, uint32_t at, uint64_t bd, uint32_t idesc, bool acc) {
+            if (CTAS == 2) ptx::mma_ts_pair(d, at, bd, idesc, acc); else ptx::mma_ts(d, at, bd, idesc, acc);
+        };
+        auto commit = [&](uint32_t bar) {      // the barrier of that name in every CTA of the item
+            if (CTAS == 2) ptx::mma_commit_pair(bar, (uint16_t)3); else ptx::mma_commit(bar);
+        };
         bool ok = true;
         auto wait_u = [&](uint32_t bar, uint32_t parity, int code) -> bool {
             return warp_wait(bar, parity, code, a.status, s_abort, lane);
         };
         // descriptors differ only in their address field (units of 16 bytes): build them once
         const uint64_t qdesc0 = make_sdesc(smem_base + kSmemQOff, 16, 1024);
-        const uint64_t kdesc0 = make_sdesc(smem_base + kSmemKOff, 16, 1024);            // K-major, 64 keys per CTA
-        const uint64_t vdesc0 = make_sdesc(smem_base + kSmemVOff, kHalfBytes, 1024);    // MN-major, 64 channels per CTA
+        const uint64_t kdesc0 = make_sdesc(smem_base + kSmemKOff, 16, 1024);            // K-major; 64 (pair) or 128 keys per CTA
+        const uint64_t vdesc0 = make_sdesc(smem_base + kSmemVOff, kHalfBytes, 1024);    // MN-major; 64-channel blocks 16 KB apart
         auto issue_s = [&](int jj) {             // S_jj = Q K_jj^T into score buffer jj % 3
             if (ptx::elect_one()) {
                 const int stage = jj % kKStages;
-                const uint64_t kd = kdesc0 + (uint64_t)((stage * kHalfBytes) >> 4);
+                const uint64_t kd = kdesc0 + (uint64_t)((stage * kStageBytes) >> 4);
                 const uint32_t d = tmem + (uint32_t)(jj % kScoreBufs) * 128;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t qoff = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
-                    const uint64_t koff = (uint64_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4);
-                    ptx::mma_ss_pair(d, qdesc0 + qoff, kd + koff, idesc_s, ks > 0);
+                    const uint64_t koff = (uint64_t)(((ks >> 2) * (kStageBytes / 2) + (ks & 3) * 32) >> 4);
+                    mma_ss(d, qdesc0 + qoff, kd + koff, idesc_s, ks > 0);
                 }
-                ptx::mma_commit_pair(bar_s_full + 8 * (jj % kScoreBufs), both);
-                ptx::mma_commit_pair(bar_k_empty + 8 * stage, both);
+                commit(bar_s_full + 8 * (jj % kScoreBufs));
+                commit(bar_k_empty + 8 * stage);
             }
         };
         auto issue_pv = [&](int jj) {            // O (+)= P_jj V_jj
             if (ptx::elect_one()) {
                 const int stage = jj % kVStages;
-                const uint64_t vd = vdesc0 + (uint64_t)((stage * kHalfBytes) >> 4);
+                const uint64_t vd = vdesc0 + (uint64_t)((stage * kStageBytes) >> 4);
                 const uint32_t p = tmem + (uint32_t)(jj % kScoreBufs) * 128;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    ptx::mma_ts_pair(tmem + kColO, p + (ks >> 1) * 32 + (ks & 1) * 8, vd + (uint64_t)((ks * 2048) >> 4),
-                                     idesc_pv, jj > 0 || ks > 0);
-                ptx::mma_commit_pair(bar_pv_done + 8 * (jj & 3), both);
-                ptx::mma_commit_pair(bar_v_empty + 8 * stage, both);
-                if (jj == ntiles - 1) ptx::mma_commit_pair(bar_o_full, both);
+                    mma_ts(tmem + kColO, p + (ks >> 1) * 32 + (ks & 1) * 8, vd + (uint64_t)((ks * 2048) >> 4),
+                           idesc_pv, jj > 0 || ks > 0);
+                commit(bar_pv_done + 8 * (jj & 3));
+                commit(bar_v_empty + 8 * stage);
+                if (jj == ntiles - 1) commit(bar_o_full);
             }
         };
 
@@ -503,7 +554,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             if (lane == 0 && jj < 8) EVLN_STAMP(34 + 3 * jj);
             __syncwarp();
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && (warp & 3) < quarters) {
         // ================= softmax + epilogue =================
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
         const int part = (warp - 4) >> 2;                  // which 32 columns of a row
@@ -516,7 +567,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int bound = row_valid ? w.L + r_local / a.G : 0x3fffffff;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
         const uint32_t t_o = t_lane + kColO + part * 32;
-        const uint32_t p_full0 = ptx::map_to_cta(bar_p_full, 0);
+        const uint32_t p_full0 = CTAS == 2 ? ptx::map_to_cta(bar_p_full, 0) : bar_p_full;
 
         float m_ref = -INFINITY;      // reference maximum (log2 domain) the exponentials use
         float l = 0.f;                // this thread's share of the running sum of exponentials
@@ -689,7 +740,9 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::tmem_st_wait();
             ptx::fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(p_full0 + 8 * buf);
+            if (lane == 0) {
+                if (CTAS == 2) ptx::mbar_arrive_cluster(p_full0 + 8 * buf); else ptx::mbar_arrive(p_full0 + 8 * buf);
+            }
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(4 + 3 * jj);
         }
 
@@ -749,13 +802,35 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // ---- teardown: nobody leaves while the other CTA may still touch this CTA's memory ----
     ptx::fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive();
-    ptx::cluster_wait();
+    if (CTAS == 2) {
+        ptx::cluster_arrive();
+        ptx::cluster_wait();
+    }
     if (warp == 1) {
         ptx::fence_after_sync();
-        ptx::tmem_dealloc_pair(tmem, 512);
+        if (CTAS == 2) ptx::tmem_dealloc_pair(tmem, 512); else ptx::tmem_dealloc(tmem, 512);
         if (lane == 0) EVLN_STAMP(62);
     }
+}
+
+// One CTA pair per work item (256 query rows): any number of rows, contiguous or paged cache.
+template <bool PAGED, typename LensT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const TcAttnArgs a,
+                 const __grid_constant__ LensT lens)
+{
+    attn_tc_body<PAGED, LensT, 2>(tm_q, tm_k, tm_v, a, lens);
+}
+
+// One CTA per work item, for steps whose rows per kv head fit one 128-row tile (the few action
+// tokens that follow a frame, Sec. 3.1): the KV range is cut into as many splits as there are SMs,
+// and each CTA streams whole K/V tiles, so the step runs at the rate HBM delivers the cache.
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_solo_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const TcAttnArgs a)
+{
+    attn_tc_body<false, NoLens, 1>(tm_q, tm_k, tm_v, a, NoLens{});
 }
 
 }  // namespace evln

@@ -132,6 +132,29 @@ int choose_splits_tc(int units_total, int nkv_max, int nkv_min, int num_sms)
     return best;
 }
 
+// A step whose rows per kv head fit one 128-row tile (a few new tokens: the action tokens after a
+// frame) runs one CTA per (kv head, split) instead of CTA pairs.
+inline bool use_solo_kernel(const evlnStepParams* p)
+{
+    return use_tensor_kernel(p) && (long)p->num_new * (p->num_q_heads / p->num_kv_heads) <= kTileM;
+}
+
+// Split schedule of the one-CTA-per-item kernel: the step is bound by streaming K/V once, so the
+// KV range is spread over all SMs; an item's fixed cost is about 3 tiles of streaming, and a split
+// adds a partial row set of R rows to merge.
+int choose_splits_solo(int Hkv, int R, int nkv, int num_sms)
+{
+    int best = 1;
+    double best_cost = 1e30;
+    const int smax = nkv < kMaxSplits ? (nkv < 1 ? 1 : nkv) : kMaxSplits;
+    for (int s = 1; s <= smax; ++s) {
+        const double waves = ceil((double)Hkv * s / num_sms);
+        const double cost = waves * (ceil((double)nkv / s) + 3.0) + 0.5 * s * R / 256.0;
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = s; }
+    }
+    return best;
+}
+
 int resolve_splits(evlnHandle_t h, const evlnStepParams* p)
 {
     if (p->num_new == 0) return 1;
@@ -139,6 +162,8 @@ int resolve_splits(evlnHandle_t h, const evlnStepParams* p)
     const int G = p->num_q_heads / p->num_kv_heads;
     const int R = p->num_new * G;
     const int T = p->cache_len + p->num_new;
+    if (use_solo_kernel(p))
+        return choose_splits_solo(p->num_kv_heads, R, ceil_div(T, kTileN), h->num_sms);
     if (use_tensor_kernel(p)) {
         const int units = ceil_div(R, kUnitRows);
         const int nkv_max = unit_kv_tiles(p->cache_len, p->num_new, G, units - 1, kUnitRows);
@@ -297,6 +322,8 @@ evlnStatus_t evlnCreate(evlnHandle_t* handle, int device)
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(attn_pair_kernel<true, BatchLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kTcSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSoloSmemBytes);
     if (e != cudaSuccess) {
         if (h->d_status) cudaFree(h->d_status);
         delete h;
@@ -426,23 +453,27 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
             cuuint64_t strides[2] = {256, (cuuint64_t)p->cache_capacity * 256};
             // per CTA of a pair: half a K tile is 64 keys x all channels (two boxes), half a V tile
             // is 128 keys x 64 channels (one box)
+            // (a CTA on its own takes whole tiles: two 128-key boxes each)
             cuuint32_t box_k[3] = {64, 64, 1};
             cuuint32_t box_v[3] = {64, 128, 1};
-            if (!encode_map(h, &tm_k, k_cache, 3, dims, strides, box_k)) return EVLN_INVALID_VALUE;
+            if (!encode_map(h, &tm_k, k_cache, 3, dims, strides, use_solo_kernel(p) ? box_v : box_k)) return EVLN_INVALID_VALUE;
             if (!encode_map(h, &tm_v, v_cache, 3, dims, strides, box_v)) return EVLN_INVALID_VALUE;
         }
         TcAttnArgs a = {};
         a.o_part = o_part; a.lse_part = lse_part; a.page_table = nullptr; a.status = h->d_status;
         a.Hkv = p->num_kv_heads; a.G = G; a.rows = R;
         a.cache_len = p->cache_len; a.num_new = p->num_new; a.num_splits = S;
-        a.units_per_head = ceil_div(R, kUnitRows);
+        a.units_per_head = use_solo_kernel(p) ? 1 : ceil_div(R, kUnitRows);
         a.scale_log2 = scale * 1.4426950408889634f;
 #ifdef EVLN_TIMELINE
         a.timeline = g_timeline;
 #endif
         NoLens nl = {};
         const int items = S * p->num_kv_heads * a.units_per_head;
-        launch_pair_pdl(attn_pair_kernel<false, NoLens>, items, kTcSmemBytes, st, tm_q, tm_k, tm_v, a, nl);
+        if (use_solo_kernel(p))
+            launch_pdl(attn_solo_kernel, dim3(items), dim3(kTcThreads), kSoloSmemBytes, st, tm_q, tm_k, tm_v, a);
+        else
+            launch_pair_pdl(attn_pair_kernel<false, NoLens>, items, kTcSmemBytes, st, tm_q, tm_k, tm_v, a, nl);
     } else {
         SimtAttnArgs a = {};
         a.q_rot = q_rot; a.k_cache = k_cache; a.v_cache = v_cache;
@@ -463,6 +494,7 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
 
+
 evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void* workspace, void* out,
                              float* lse_out, void* stream)
 {
@@ -481,6 +513,27 @@ evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16) return launch_combine<__nv_bfloat16>(h, a, p->head_dim, false, nullptr, st);
     return launch_combine<float>(h, a, p->head_dim, false, nullptr, st);
+}
+
+evlnStatus_t evlnStep(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
+                      const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok, void* q_rot,
+                      void* k_cache, void* v_cache, void* workspace, size_t workspace_bytes, void* out,
+                      float* lse_out, void* stream)
+{
+    evlnStatus_t s = check_step_params(h, p);
+    if (s != EVLN_OK) return s;
+    if (p->num_new == 0) return EVLN_OK;
+    // every argument is checked before the first launch, so a rejected call has done nothing
+    if (!workspace || !out || !aligned16(workspace) || !aligned16(out)) return EVLN_INVALID_VALUE;
+    const long rows = (long)p->num_new * (p->num_q_heads / p->num_kv_heads);
+    if (workspace_bytes < partial_bytes(resolve_splits(h, p), p->num_kv_heads, rows, p->head_dim))
+        return EVLN_WORKSPACE_TOO_SMALL;
+    s = evlnRopeAppend(h, p, q_new, k_new, v_new, q_stride_tok, k_stride_tok, v_stride_tok, q_rot, k_cache, v_cache,
+                       stream);
+    if (s != EVLN_OK) return s;
+    s = evlnStepAttention(h, p, q_rot, k_cache, v_cache, workspace, workspace_bytes, stream);
+    if (s != EVLN_OK) return s;
+    return evlnStepCombine(h, p, workspace, out, lse_out, stream);
 }
 
 // ---- paged -------------------------------------------------------------------------------
@@ -787,6 +840,8 @@ evlnStatus_t noalloc_setup(int device, NoAllocDevice** out)
         if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return EVLN_CUDA_ERROR;
         e = cudaFuncSetAttribute(attn_pair_kernel<false, NoLens>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kTcSmemBytes);
+        if (e != cudaSuccess) return EVLN_CUDA_ERROR;
+        e = cudaFuncSetAttribute(attn_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSoloSmemBytes);
         if (e != cudaSuccess) return EVLN_CUDA_ERROR;
         d->ctx.device = device;
         d->ctx.num_sms = prop.multiProcessorCount;

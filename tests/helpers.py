@@ -28,7 +28,7 @@ class GpuStep:
     """Device buffers of one layer + the three calls of a step, all through the C-ABI."""
 
     def __init__(self, handle, dtype, Hq, Hkv, D, capacity, theta, max_new, scale=0.0,
-                 num_splits=0, kernel=B.EVLN_KERNEL_AUTO, device="cuda:0"):
+                 num_splits=0, kernel=B.EVLN_KERNEL_AUTO, device="cuda:0", fused=False):
         self.h, self.dtype, self.Hq, self.Hkv, self.D = handle, dtype, Hq, Hkv, D
         self.cap, self.theta, self.scale = capacity, theta, scale
         self.num_splits, self.kernel = num_splits, kernel
@@ -38,6 +38,7 @@ class GpuStep:
         self.k_cache = torch.full((Hkv, capacity, D), 7.0, dtype=self.tdt, device=device)
         self.v_cache = torch.full((Hkv, capacity, D), -3.0, dtype=self.tdt, device=device)
         self.max_new = max_new
+        self.fused = fused        # evlnStep instead of the three calls
 
     def load_cache(self, k_tok_major, v_tok_major):
         L = k_tok_major.shape[0]
@@ -56,9 +57,12 @@ class GpuStep:
         ws = torch.empty(max(B.evlnStepWorkspaceSize(self.h, p), 16), dtype=torch.uint8, device=self.dev)
         out = torch.full((n, self.Hq, self.D), float("nan"), dtype=self.tdt, device=self.dev)
         lse = torch.full((n, self.Hq), float("nan"), dtype=torch.float32, device=self.dev)
-        B.evlnRopeAppend(self.h, p, q_new, k_new, v_new, q_rot, self.k_cache, self.v_cache)
-        B.evlnStepAttention(self.h, p, q_rot, self.k_cache, self.v_cache, ws)
-        B.evlnStepCombine(self.h, p, ws, out, lse)
+        if self.fused:
+            B.evlnStep(self.h, p, q_new, k_new, v_new, q_rot, self.k_cache, self.v_cache, ws, out, lse)
+        else:
+            B.evlnRopeAppend(self.h, p, q_new, k_new, v_new, q_rot, self.k_cache, self.v_cache)
+            B.evlnStepAttention(self.h, p, q_rot, self.k_cache, self.v_cache, ws)
+            B.evlnStepCombine(self.h, p, ws, out, lse)
         status = B.evlnGetDeviceStatus(self.h)
         assert status == 0, f"device status {status}: a bounded wait expired"
         G = self.Hq // self.Hkv

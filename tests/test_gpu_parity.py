@@ -128,6 +128,80 @@ def test_tc_kernel_reference_moves_in_late_tiles(handle):
         _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
 
 
+# ---- few new tokens: one CTA per (kv head, split) --------------------------------------------
+
+@pytest.mark.parametrize("L,n,splits", [
+    (4096, 8, 0),         # an action chunk after a frame, schedule chosen by the library
+    (4096, 1, 0),         # one token
+    (20656, 8, 0),        # end of a 100-step episode
+    (4090, 8, 0),         # the new tokens straddle two KV tiles
+    (1000, 18, 4),        # 126 rows: the most one tile takes
+    (1000, 19, 3),        # 133 rows: back on CTA pairs
+    (130, 4, 2),          # one tile per split
+    (0, 3, 1),            # no history at all
+    (300, 16, 9),         # more splits than KV tiles: empty splits
+    (257, 5, 0),          # rows in the first lane quarter only
+    (3000, 10, 32),       # the largest split count
+])
+def test_tc_kernel_few_new_tokens(handle, L, n, splits):
+    cfg = dataclasses.replace(W.STEP_7B, name=f"few_{L}_{n}", cache_len=L, num_new=n, seed=300 + L + n)
+    _run(handle, cfg, num_splits=splits)
+
+
+def test_few_new_tokens_reference_moves(handle):
+    # as test_tc_kernel_reference_moves_in_late_tiles, on the one-CTA kernel with idle lane quarters
+    cfg = dataclasses.replace(W.STEP_7B, name="few_moves", cache_len=1700, num_new=8, input_scale=1.0, seed=12)
+    x = W.make_step_inputs(cfg)
+    x["k_cache"][700] *= 48.0
+    x["k_cache"][1410:1412] *= 128.0
+    x["k_new"][5] *= 250.0
+    for splits in (1, 2):
+        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
+
+
+@pytest.mark.parametrize("L,n", [(4096, 196), (4096, 8), (700, 130), (2000, 1)])
+def test_fused_step_call_is_bitwise_the_three_calls(handle, L, n):
+    cfg = dataclasses.replace(W.STEP_7B, name=f"fused_{L}_{n}", cache_len=L, num_new=n, seed=400 + n)
+    x = W.make_step_inputs(cfg)
+    res = []
+    for fused in (False, True):
+        gs = GpuStep(handle, "bf16", cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n + 5, cfg.rope_theta, n,
+                     fused=fused)
+        gs.load_cache(x["k_cache"], x["v_cache"])
+        g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
+        res.append((g, gs))
+    (a, gsa), (b, gsb) = res
+    assert torch.equal(a["out"].view(torch.int16), b["out"].view(torch.int16))
+    assert torch.equal(a["lse"], b["lse"])
+    assert torch.equal(gsa.k_cache.view(torch.int16), gsb.k_cache.view(torch.int16))
+    assert torch.equal(gsa.v_cache.view(torch.int16), gsb.v_cache.view(torch.int16))
+    r = oracle_step("bf16", x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L, cfg.rope_theta)
+    check_output("bf16", b["out"], b["lse"], r["out"], r["lse"])
+
+
+def test_fused_step_calls_in_a_chain(handle):
+    # frame step, action step, next frame at the same length (the action keys are overwritten),
+    # all through the one-call form back to back on one stream
+    Hq, Hkv, D, theta = 28, 4, 128, 1.0e6
+    I, F, A, N = 100, 196, 8, 4
+    gen = torch.Generator().manual_seed(77)
+    mk = lambda n, H, sc: (torch.randn((n, H, D), generator=gen) * sc).to(torch.bfloat16)
+    cap = I + N * F + A
+    gs = GpuStep(handle, "bf16", Hq, Hkv, D, cap, theta, F, fused=True)
+    kc, vc = np.zeros((cap, Hkv, D)), np.zeros((cap, Hkv, D))
+    L = 0
+    steps = [(I, True)]
+    for _ in range(N):
+        steps += [(F, True), (A, False)]
+    for n, keep in steps:
+        q, k, v = mk(n, Hq, 0.3), mk(n, Hkv, 0.3), mk(n, Hkv, 1.0)
+        g = gs.step(L, q, k, v)
+        r = so.step(f64(q), f64(k), f64(v), kc, vc, L, theta, 0.0, storage="bf16")
+        check_output("bf16", g["out"], g["lse"], r["out"], r["lse"])
+        if keep:
+            L += n
+
+
 def test_tc_matches_simt_kernel_on_device(handle):
     cfg = dataclasses.replace(W.STEP_7B, name="cross", cache_len=700, num_new=90, seed=8)
     a, _ = _run(handle, cfg)
