@@ -253,7 +253,7 @@ def run_ours(args, rank, world, local_rank, dist):
     # a short measurement each, on rank 0 of a single-GPU run only.
     h2d = sum(t.numel() * t.element_size() for t in ring.layers[0]["host_in"])
     d2h = ring.layers[0]["host_out"].numel() * ring.layers[0]["host_out"].element_size()
-    by_len = []
+    by_len, action_steps = [], []
     if world == 1 and not args.no_sweep:
         del g_step, g_attn
         ring.layers.clear()
@@ -275,6 +275,23 @@ def run_ours(args, rank, world, local_rank, dist):
                            "attention_tflops": round(c.flops() / t_a / 1e6, 1), "kv_splits": r.splits,
                            "step_roofline_frac": round(roof / t_s, 4)})
             del gs, ga, r
+            torch.cuda.empty_cache()
+        # The 8 action tokens that follow a frame in the streaming episode (same layer shape): a step
+        # bound by streaming K and V once, quoted against the measured HBM bandwidth.
+        for L in (4096, 20656):
+            c = dataclasses.replace(cfg, name=f"action_7b_L{L}", cache_len=L, num_new=8)
+            kv_bytes = 2 * (L + c.num_new) * c.num_kv_heads * c.head_dim * 2
+            layers = max(2, min(RING_LAYERS, int(2.2 * L2_BYTES / kv_bytes) + 1))
+            r = LayerRing(B, handle, c, dev, layers, random_device_inputs=True)
+            gs = capture(r.step, layers)
+            reps = max(3, 640 // layers)
+            for _ in range(3):
+                gs.replay()
+            t_s = timed(gs.replay, reps, barrier) * 1e3 / (reps * layers)
+            action_steps.append({"cache_len": L, "new_tokens": 8, "us_per_step": round(t_s, 2), "kv_splits": r.splits,
+                                 "kv_gbs": round(kv_bytes / t_s / 1e3, 1),
+                                 "hbm_frac": round(kv_bytes / t_s / 1e3 / peaks_s["hbm_gbs"], 4)})
+            del gs, r
             torch.cuda.empty_cache()
         assert B.evlnGetDeviceStatus(handle) == 0, "a kernel gave up on a bounded wait"
     B.evlnDestroy(handle)
@@ -320,6 +337,8 @@ def run_ours(args, rank, world, local_rank, dist):
     }
     if by_len:
         line["by_cache_len"] = by_len
+    if action_steps:
+        line["action_token_step"] = action_steps
     return line
 
 

@@ -27,11 +27,11 @@ def handle():
 
 
 def _run(handle, cfg, kernel=B.EVLN_KERNEL_AUTO, num_splits=0, extra_cap=37, lse_tol=1e-3, rel_tol=1e-2,
-         inputs=None, round_q=False, abs_tol=1e-2):
+         inputs=None, round_q=False, abs_tol=1e-2, fused=False):
     x = inputs or W.make_step_inputs(cfg)
     L, n = cfg.cache_len, cfg.num_new
     gs = GpuStep(handle, cfg.dtype, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n + extra_cap,
-                 cfg.rope_theta, n, num_splits=num_splits, kernel=kernel)
+                 cfg.rope_theta, n, num_splits=num_splits, kernel=kernel, fused=fused)
     gs.load_cache(x["k_cache"], x["v_cache"])
     g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
     r = oracle_step(cfg.dtype, x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L,
@@ -148,6 +148,15 @@ def test_tc_kernel_few_new_tokens(handle, L, n, splits):
     _run(handle, cfg, num_splits=splits)
 
 
+@pytest.mark.parametrize("L,n,splits", [
+    (4096, 8, 0), (4096, 1, 0), (20656, 8, 0), (4090, 8, 0), (4095, 2, 5), (1000, 18, 4), (130, 4, 2), (0, 3, 1),
+    (300, 16, 9), (257, 5, 0), (3000, 10, 32), (3000, 10, 1), (127, 1, 0), (128, 1, 0),
+])
+def test_one_call_step_of_few_new_tokens(handle, L, n, splits):
+    cfg = dataclasses.replace(W.STEP_7B, name=f"one_{L}_{n}", cache_len=L, num_new=n, seed=500 + L + n)
+    _run(handle, cfg, num_splits=splits, fused=True)
+
+
 def test_few_new_tokens_reference_moves(handle):
     # as test_tc_kernel_reference_moves_in_late_tiles, on the one-CTA kernel with idle lane quarters
     cfg = dataclasses.replace(W.STEP_7B, name="few_moves", cache_len=1700, num_new=8, input_scale=1.0, seed=12)
@@ -157,9 +166,11 @@ def test_few_new_tokens_reference_moves(handle):
     x["k_new"][5] *= 250.0
     for splits in (1, 2):
         _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
+        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2,
+             fused=True)
 
 
-@pytest.mark.parametrize("L,n", [(4096, 196), (4096, 8), (700, 130), (2000, 1)])
+@pytest.mark.parametrize("L,n", [(4096, 196), (4096, 8), (700, 130), (2000, 1), (4090, 8), (20656, 8)])
 def test_fused_step_call_is_bitwise_the_three_calls(handle, L, n):
     cfg = dataclasses.replace(W.STEP_7B, name=f"fused_{L}_{n}", cache_len=L, num_new=n, seed=400 + n)
     x = W.make_step_inputs(cfg)
