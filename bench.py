@@ -111,6 +111,27 @@ def physical_gpu_index(local_index: int) -> int:
 # our arm
 # ------------------------------------------------------------------------------------------------
 
+# DRAM bytes (read + write) of one attention launch at this workload, from the ncu capture that
+# profiles/attn_pair_kernel_step_7b_L4096.md summarises.  The counters belong to the kernel sources
+# as they were then: once one of them changes, the figure is withheld until it is taken again.
+K2_DRAM_BYTES_PER_LAUNCH = 10_255_872
+K2_SOURCES = ("attn_pair.cuh", "ptx_sm100.cuh", "common.cuh")
+K2_SOURCES_SHA256 = "aff42e08ef7bed7c0a0cafe8a58769f5c1cc5d6aaae98b8d22185a152dd042fc"
+
+
+def attention_dram_traffic():
+    import hashlib
+    h = hashlib.sha256()
+    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2512_10310_b200", "csrc")
+    try:
+        for name in K2_SOURCES:
+            with open(os.path.join(src, name), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return K2_DRAM_BYTES_PER_LAUNCH if h.hexdigest() == K2_SOURCES_SHA256 else None
+
+
 class LayerRing:
     """Device buffers of RING_LAYERS independent layers of the workload + pinned host copies."""
 
@@ -326,7 +347,7 @@ def run_ours(args, rank, world, local_rank, dist):
             "kernel": "attn_pair_kernel (evlnStepAttention)", "bound": "tensor",
             "achieved": round(achieved_tf, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
             "frac": round(achieved_tf / peaks["bf16_tflops"], 4), "peak_kind": f"{peaks_kind} burst bf16",
-            "traffic": None, "us_per_launch": round(us_attn, 3),
+            "traffic": attention_dram_traffic(), "us_per_launch": round(us_attn, 3),
             "timing": f"CUDA events around graph replays of {RING_LAYERS} back-to-back attention launches",
             "flops_per_launch": flops,
         },
