@@ -91,20 +91,36 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
 #pragma unroll
         for (int c = 0; c < C; ++c) acc[c] = fmaf(ws, pre[s][c], acc[c]);
     }
-    for (int s = kPre; s < S; ++s) {
-        const float ws = __shfl_sync(0xffffffffu, w, s);
-        if (ws == 0.f) continue;                               // uniform across the warp
-        const float* op = a.o_part + (prow0 + s * stride_s) * D + lane * C;
-        float v[C];
-        if (C == 4) {
-            float4 x = *reinterpret_cast<const float4*>(op);
-            v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
-        } else {
+    // the remaining splits four at a time: their loads are in flight together, the sums keep the
+    // order of the splits
+    constexpr int kBatch = 8;
+    for (int s0 = kPre; s0 < S; s0 += kBatch) {
+        float v[kBatch][C];
 #pragma unroll
-            for (int c = 0; c < C; ++c) v[c] = op[c];
+        for (int k = 0; k < kBatch; ++k) {
+            const int s = s0 + k;
+            if (s < S) {
+                const float* op = a.o_part + (prow0 + s * stride_s) * D + lane * C;
+                if (C == 4) {
+                    float4 x = *reinterpret_cast<const float4*>(op);
+                    v[k][0] = x.x; v[k][1] = x.y; v[k][2] = x.z; v[k][3] = x.w;
+                } else {
+#pragma unroll
+                    for (int c = 0; c < C; ++c) v[k][c] = op[c];
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < C; ++c) v[k][c] = 0.f;
+            }
         }
 #pragma unroll
-        for (int c = 0; c < C; ++c) acc[c] = fmaf(ws, v[c], acc[c]);
+        for (int k = 0; k < kBatch; ++k) {
+            const float ws = (s0 + k < S) ? __shfl_sync(0xffffffffu, w, s0 + k) : 0.f;   // 0 for empty splits too
+            if (ws != 0.f) {                                                            // uniform across the warp
+#pragma unroll
+                for (int c = 0; c < C; ++c) acc[c] = fmaf(ws, v[k][c], acc[c]);
+            }
+        }
     }
     const float inv = (wsum > 0.f) ? 1.f / wsum : 0.f;
 
