@@ -213,15 +213,17 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
     WorkItem w;
     if (!PAGED) {
         w.b = 0;
-        w.unit = item % a.units_per_head;
-        w.g = (item / a.units_per_head) % a.Hkv;
-        w.slot = item / (a.units_per_head * a.Hkv);
+        // (unsigned 32-bit arithmetic throughout: see unit_kv_tiles)
+        const unsigned per_head = (unsigned)item / (unsigned)a.units_per_head;
+        w.unit = (int)((unsigned)item - per_head * (unsigned)a.units_per_head);
+        w.slot = (int)(per_head / (unsigned)a.Hkv);
+        w.g = (int)(per_head - (unsigned)w.slot * (unsigned)a.Hkv);
         w.L = a.cache_len;
         w.n = a.num_new;
         w.row_base = 0;
         const int nkv = unit_kv_tiles(w.L, w.n, a.G, w.unit, UNIT_ROWS);
-        w.j0 = (int)((long)w.slot * nkv / a.num_splits);
-        w.j1 = (int)((long)(w.slot + 1) * nkv / a.num_splits);
+        w.j0 = (int)((unsigned)w.slot * (unsigned)nkv / (unsigned)a.num_splits);
+        w.j1 = (int)((unsigned)(w.slot + 1) * (unsigned)nkv / (unsigned)a.num_splits);
     } else {
         int rem = item;
         int b = 0;
@@ -380,7 +382,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     ptx::fence_before_sync();
     __syncthreads();
     if (CTAS == 2) {
-        ptx::cluster_arrive();  // the other CTA's barriers exist before anything arrives on them
+        // the other CTA's barriers exist before anything arrives on them (their initialisation was
+        // released cluster-wide by fence.mbarrier_init; nothing else is shared yet)
+        ptx::cluster_arrive_relaxed();
         ptx::cluster_wait();
     }
     ptx::fence_after_sync();
@@ -803,7 +807,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     ptx::fence_before_sync();
     __syncthreads();
     if (CTAS == 2) {
-        ptx::cluster_arrive();
+        // every cross-CTA signal and tensor-memory access of the item is behind the last commit both
+        // CTAs waited for; this meeting only keeps either CTA from freeing the pair's tensor memory early
+        ptx::cluster_arrive_relaxed();
         ptx::cluster_wait();
     }
     if (warp == 1) {

@@ -44,10 +44,12 @@ __device__ __forceinline__ void from_float(float x, __nv_bfloat16& y) { y = __fl
 // Number of 128-key tiles the rows of unit u (rows [u*unit_rows, ...)) of an episode need.
 __host__ __device__ inline int unit_kv_tiles(int L, int n, int G, int unit, int unit_rows)
 {
-    long last_row = (long)(unit + 1) * unit_rows - 1;
-    long last_tok = last_row / G;
-    if (last_tok > n - 1) last_tok = n - 1;
-    return (int)((L + last_tok + 1 + kTileN - 1) / kTileN);
+    // 32-bit on purpose (rows per kv head are at most 2^24): a 64-bit division costs a CTA hundreds
+    // of cycles before it has started anything
+    unsigned last_row = (unsigned)(unit + 1) * (unsigned)unit_rows - 1u;
+    unsigned last_tok = last_row / (unsigned)G;
+    if (last_tok > (unsigned)(n - 1)) last_tok = (unsigned)(n - 1);
+    return (int)(((unsigned)L + last_tok + 1u + (unsigned)kTileN - 1u) / (unsigned)kTileN);
 }
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -233,6 +233,13 @@ __device__ __forceinline__ void cluster_arrive()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 }
+// arrival without the cluster-wide release of this thread's earlier writes (a flush that costs about
+// a thousand cycles): for meetings whose only shared state is ordered by fences of its own
+// (fence.mbarrier_init for the barriers, tcgen05 fences for tensor memory)
+__device__ __forceinline__ void cluster_arrive_relaxed()
+{
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void cluster_wait()
 {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
