@@ -625,6 +625,8 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         // (a power-of-two factor, exact): running sum, its channels of O, and its parts of the P
         // tiles that are written but not yet consumed.
         int nrare = 0;                // meetings on bar_rare so far
+        bool sum_published = false;   // this thread's share of the row sum is out for the final exchange
+        float* s_sum = s_xch + kParts * 128;
         auto move_reference = [&](int released, bool mine, float want) -> bool {
             s_cand[part * 128 + r_tile] = mine ? want : m_ref;
             if (lane == 0) s_rel[quarter * kParts + part] = released;
@@ -685,6 +687,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 ptx::fence_before_sync();
             }
             m_ref = m_new;
+            if (sum_published) s_sum[part * 128 + r_tile] = l;     // (ordered by the meeting below)
             return meet(bar_rare, nrare++);
         };
 
@@ -750,26 +753,29 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(4 + 3 * jj);
         }
 
-        // all tiles handed over; a slower warp of the quarter may still ask for a new reference
+        // All tiles handed over.  The row sum is the sum over the row's threads (same reference in
+        // all): they exchange it while the last product is still running.  A slower warp of the quarter
+        // may still ask for a new reference until it arrives here too; whoever serves such a request
+        // after publishing its share publishes the rescaled share again (inside move_reference).
+        if (ok) {
+            s_sum[part * 128 + r_tile] = l;
+            sum_published = true;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
+        }
         while (ok) {
-            const int r = wait_or_request(bar_o_full, 0, kDevTimeoutSoftmaxO);
+            const int r = wait_or_request(bar_xch + 8 * quarter, 1, kDevTimeoutSoftmaxX);
             if (r == 0) break;
             ok = (r == 1) && move_reference(ntiles, false, 0.f);
         }
-
+        // nobody of the quarter can ask any more; the last product
+        if (ok) ok = warp_wait(bar_o_full, 0, kDevTimeoutSoftmaxO, a.status, s_abort, lane);
         if (ok) {
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(60);
-            // the row sum is the sum over the row's threads (same reference in all)
-            float* xch = s_xch + kParts * 128;
-            xch[part * 128 + r_tile] = l;
-            ok = meet(bar_xch, 1);
-        }
-        if (ok) {
-            const float* xch = s_xch + kParts * 128;
             l = 0.f;
 #pragma unroll
-            for (int c = 0; c < kParts; ++c) l += xch[c * 128 + r_tile];
+            for (int c = 0; c < kParts; ++c) l += s_sum[c * 128 + r_tile];
             // Epilogue: O/l goes out through shared memory so that global stores are whole
             // 128-byte lines.  The K ring is dead (its last consumer has completed); each warp
             // stages its 32 rows x 32 channels there, rows 144 bytes apart.

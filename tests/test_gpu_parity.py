@@ -122,6 +122,7 @@ def test_tc_kernel_reference_moves_in_late_tiles(handle):
     x["k_cache"][700] *= 48.0
     x["k_cache"][1410:1412] *= 128.0
     x["k_new"][50] *= 250.0
+    x["k_new"][95] *= 400.0       # the very last key: its rows' threads are already exchanging their sums
     # the winning scores are several hundred: fp32 accumulation on the tensor core resolves them to
     # a few 1e-5 relative, which is what the log-sum-exp gate allows here
     for splits in (1, 2):
@@ -164,6 +165,7 @@ def test_few_new_tokens_reference_moves(handle):
     x["k_cache"][700] *= 48.0
     x["k_cache"][1410:1412] *= 128.0
     x["k_new"][5] *= 250.0
+    x["k_new"][7] *= 400.0
     for splits in (1, 2):
         _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
         _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2,
