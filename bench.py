@@ -114,9 +114,9 @@ def physical_gpu_index(local_index: int) -> int:
 # DRAM bytes (read + write) of one attention launch at this workload, from the ncu capture that
 # profiles/attn_pair_kernel_step_7b_L4096.md summarises.  The counters belong to the kernel sources
 # as they were then: once one of them changes, the figure is withheld until it is taken again.
-K2_DRAM_BYTES_PER_LAUNCH = 10_253_056
+K2_DRAM_BYTES_PER_LAUNCH = 10_252_800
 K2_SOURCES = ("attn_pair.cuh", "ptx_sm100.cuh", "common.cuh")
-K2_SOURCES_SHA256 = "aeb8fa6589f0f1eb26d24721552a0d5a654ca514f72d5c7826a77e50a56f6a11"
+K2_SOURCES_SHA256 = "6f7c38c01567322f232d5812107eed20469ee785406c52cd6ea74afc6b542220"
 
 
 def attention_dram_traffic():
