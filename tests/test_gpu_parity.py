@@ -215,6 +215,42 @@ def test_fused_step_calls_in_a_chain(handle):
             L += n
 
 
+@pytest.mark.parametrize("n", [196, 8])
+def test_strided_views_of_a_fused_qkv_buffer(handle, n):
+    # q, k and v as the three views of one [n, Hq + 2 Hkv, D] buffer (token stride 36 * 128 elements)
+    cfg = dataclasses.replace(W.STEP_7B, name=f"fusedqkv_{n}", cache_len=1500, num_new=n, seed=600 + n)
+    x = W.make_step_inputs(cfg)
+    Hq, Hkv, D, L = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.cache_len
+    qkv = torch.cat([x["q_new"], x["k_new"], x["v_new"]], dim=1).contiguous().to("cuda:0")
+    q, k, v = qkv[:, :Hq], qkv[:, Hq:Hq + Hkv], qkv[:, Hq + Hkv:]
+    assert not q.is_contiguous() and q.stride(0) == (Hq + 2 * Hkv) * D
+    gs = GpuStep(handle, "bf16", Hq, Hkv, D, L + n, cfg.rope_theta, n)
+    gs.load_cache(x["k_cache"], x["v_cache"])
+    p = gs.params(L, n)
+    q_rot = torch.empty(B.evlnStepQRotSize(handle, p), dtype=torch.uint8, device="cuda:0")
+    ws = torch.empty(max(B.evlnStepWorkspaceSize(handle, p), 16), dtype=torch.uint8, device="cuda:0")
+    out = torch.full((n, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+    lse = torch.full((n, Hq), float("nan"), dtype=torch.float32, device="cuda:0")
+    B.evlnStep(handle, p, q, k, v, q_rot, gs.k_cache, gs.v_cache, ws, out, lse)
+    assert B.evlnGetDeviceStatus(handle) == 0
+    r = oracle_step("bf16", x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L, cfg.rope_theta)
+    check_cache(gs, r, L, n)
+    check_output("bf16", out, lse, r["out"], r["lse"])
+
+
+def test_one_call_step_fp32(handle):
+    # the one-call form on the fp32 configuration (SIMT attention kernel)
+    cfg = W.TINY_F32
+    x = W.make_step_inputs(cfg)
+    L, n = cfg.cache_len, cfg.num_new
+    gs = GpuStep(handle, "f32", cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n, cfg.rope_theta, n, fused=True)
+    gs.load_cache(x["k_cache"], x["v_cache"])
+    g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
+    r = oracle_step("f32", x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L, cfg.rope_theta)
+    check_cache(gs, r, L, n)
+    check_output("f32", g["out"], g["lse"], r["out"], r["lse"])
+
+
 def test_tc_matches_simt_kernel_on_device(handle):
     cfg = dataclasses.replace(W.STEP_7B, name="cross", cache_len=700, num_new=90, seed=8)
     a, _ = _run(handle, cfg)
