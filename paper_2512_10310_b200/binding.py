@@ -16,7 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "lib", "libevln.so")
 _SOURCES = ["evln_api.cu", "attn_pair.cuh", "attn_simt.cuh", "combine.cuh", "rope_append.cuh",
-            "common.cuh", "ptx_sm100.cuh", "gather_rope.cuh"]
+            "common.cuh", "ptx_sm100.cuh", "gather_rope.cuh", "timeline_debug.cuh"]
 
 EVLN_OK, EVLN_INVALID_VALUE, EVLN_NOT_SUPPORTED, EVLN_CACHE_FULL = 0, 1, 2, 3
 EVLN_WORKSPACE_TOO_SMALL, EVLN_CUDA_ERROR, EVLN_DEVICE_TIMEOUT = 4, 5, 6

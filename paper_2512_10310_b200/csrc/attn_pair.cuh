@@ -20,17 +20,23 @@
 //               buffers, O += P_j V_j (A = P from TMEM).  Scores run up to three tiles ahead
 //               of the softmax, so the tensor pipe and the softmax warps only meet through
 //               full/empty barriers and neither waits for the other's latency.
-//   warps 4-19  softmax + epilogue: thread (row, part) owns 32 of the 128 score columns of a
-//               row, so every SM sub-partition has four softmax warps whose barrier, TMEM and
-//               special-function latencies (each 100-200 cycles) hide one another.  The four
-//               threads of a row fix the row's reference maximum together on the first tile and
-//               talk to each other again only if a later score exceeds it by more than 2^64
-//               (then O, the row sums and the pending P tiles are rescaled by a power of two);
-//               the final division by the row sum makes any reference exact.  P is written
-//               back over the scores as packed bf16.
-//   warps 2-3   idle.
+//   warps 4-19  softmax + epilogue, four warps per TMEM lane quarter (= per SM sub-partition).
+//               They work in two groups on ALTERNATE KV tiles: the warps of group 0 take the
+//               even tiles of the item, those of group 1 the odd ones, and within a group a
+//               thread owns 64 of the 128 score columns of its row (two blocks of 32).  The two
+//               groups of a sub-partition are therefore half a tile period apart: while one waits
+//               for scores, reads tensor memory or hands over P, the other keeps the 4 SFU lanes
+//               busy with exponentials (a tile's 128x128 exponentials take as long as its MMAs,
+//               so that unit must not idle).  The exponentials of a row are taken against a
+//               reference that one thread of the row reads off the first 32 scores of the first
+//               tile and passes to the other three through shared memory; the threads talk to each
+//               other again only if a later score exceeds it by more than 2^64 (then O, the row
+//               sums and the pending P tiles are rescaled by a power of two); the final division
+//               by the row sum makes any reference exact.  P is written back over the scores as
+//               packed bf16.
+//   warps 2-3   set up the barriers, then idle.
 // TMEM columns: S_b at 128*b, b = 0..2; P_b (packed bf16) sits in columns [32c, 32c+16), c = 0..3,
-// of S_b, each part over the score columns of the thread that writes it; O at 384.
+// of S_b, each block over the score columns of the thread that writes it; O at 384.
 //
 // Every mbarrier wait is bounded: on expiry the CTA records a code in the device status word and
 // raises a shared abort flag; all roles then leave their loops, TMEM is freed and the pair
@@ -41,14 +47,9 @@
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "timeline_debug.cuh"
 
 namespace evln {
-
-#ifdef EVLN_TIMELINE
-#define EVLN_STAMP(slot) do { if (a.timeline && (slot) < 64) a.timeline[(long)blockIdx.x * 64 + (slot)] = clock64(); } while (0)
-#else
-#define EVLN_STAMP(slot) do { } while (0)
-#endif
 
 constexpr int kTcThreads = 640;
 constexpr int kParts = 4;                             // threads per score row (32 columns each)
@@ -98,9 +99,8 @@ struct TcAttnArgs {
     int units_per_head;       // contiguous only
     int batch, max_pages, chunk_tiles;   // paged only
     float scale_log2;         // softmax scale * log2(e)
-#ifdef EVLN_TIMELINE
-    long long* timeline;      // debug builds only: 64 clock stamps per CTA
-#endif
+    FastDiv div_g;            // division by G
+    FastDiv div_s;            // contiguous only: division by num_splits
 };
 
 // --- descriptors --------------------------------------------------------------------------
@@ -207,56 +207,58 @@ struct WorkItem {
     int j0, j1;               // KV tile range
 };
 
-template <bool PAGED, typename LensT, int UNIT_ROWS>
-__device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT& lens, int item)
+// Contiguous cache: the grid is (CTAS * units, kv heads, splits), so a CTA reads its work item off
+// its block index; the two divisions left (by G and by the split count) are multiplications by
+// constants the host prepared.  Paged batch: items are numbered episode by episode (kv head, unit,
+// split inside), the host passes the first item of every episode and the CTA searches that table.
+template <bool PAGED, typename LensT, int CTAS>
+__device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT& lens)
 {
+    constexpr int UNIT_ROWS = CTAS * kTileM;
     WorkItem w;
     if (!PAGED) {
         w.b = 0;
-        // (unsigned 32-bit arithmetic throughout: see unit_kv_tiles)
-        const unsigned per_head = (unsigned)item / (unsigned)a.units_per_head;
-        w.unit = (int)((unsigned)item - per_head * (unsigned)a.units_per_head);
-        w.slot = (int)(per_head / (unsigned)a.Hkv);
-        w.g = (int)(per_head - (unsigned)w.slot * (unsigned)a.Hkv);
+        w.unit = CTAS == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+        w.g = (int)blockIdx.y;
+        w.slot = (int)blockIdx.z;
         w.L = a.cache_len;
         w.n = a.num_new;
         w.row_base = 0;
-        const int nkv = unit_kv_tiles(w.L, w.n, a.G, w.unit, UNIT_ROWS);
-        w.j0 = (int)((unsigned)w.slot * (unsigned)nkv / (unsigned)a.num_splits);
-        w.j1 = (int)((unsigned)(w.slot + 1) * (unsigned)nkv / (unsigned)a.num_splits);
+        const uint32_t nkv = (uint32_t)unit_kv_tiles_fast(w.L, w.n, a.div_g, w.unit, UNIT_ROWS);
+        w.j0 = (int)fast_div((uint32_t)w.slot * nkv, a.div_s);
+        w.j1 = (int)fast_div((uint32_t)(w.slot + 1) * nkv, a.div_s);
     } else {
-        int rem = item;
-        int b = 0;
-        for (; b < a.batch; ++b) {
-            const int n_b = lens.new_off[b + 1] - lens.new_off[b];
-            const int units = ceil_div(n_b * a.G, UNIT_ROWS);
-            int per_head = 0;
-            for (int u = 0; u < units; ++u)
-                per_head += ceil_div(unit_kv_tiles(lens.cache_len[b], n_b, a.G, u, UNIT_ROWS), a.chunk_tiles);
-            if (rem < per_head * a.Hkv) {
-                w.b = b;
-                w.L = lens.cache_len[b];
-                w.n = n_b;
-                w.row_base = lens.new_off[b] * a.G;
-                w.g = rem / per_head;
-                rem -= w.g * per_head;
-                for (int u = 0; u < units; ++u) {
-                    const int nkv = unit_kv_tiles(w.L, n_b, a.G, u, UNIT_ROWS);
-                    const int S = ceil_div(nkv, a.chunk_tiles);
-                    if (rem < S) {
-                        w.unit = u;
-                        w.slot = rem;
-                        w.j0 = (int)((long)rem * nkv / S);
-                        w.j1 = (int)((long)(rem + 1) * nkv / S);
-                        break;
-                    }
-                    rem -= S;
-                }
+        const int item = (int)(blockIdx.x >> 1);
+        int lo = 0, hi = a.batch;             // largest b with item_off[b] <= item
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (lens.item_off[mid] <= item) lo = mid; else hi = mid;
+        }
+        const int b = lo;
+        w.b = b;
+        w.L = lens.cache_len[b];
+        w.n = lens.new_off[b + 1] - lens.new_off[b];
+        w.row_base = lens.new_off[b] * a.G;
+        w.g = w.unit = w.slot = 0;
+        w.j0 = w.j1 = 0;
+        const int per_head = (lens.item_off[b + 1] - lens.item_off[b]) / a.Hkv;
+        int rem = item - lens.item_off[b];
+        if (item >= lens.item_off[a.batch] || per_head <= 0) { w.b = -1; return w; }
+        w.g = rem / per_head;
+        rem -= w.g * per_head;
+        const int units = ceil_div(w.n * a.G, UNIT_ROWS);
+        for (int u = 0; u < units; ++u) {
+            const int nkv = unit_kv_tiles_fast(w.L, w.n, a.div_g, u, UNIT_ROWS);
+            const int S = ceil_div(nkv, a.chunk_tiles);
+            if (rem < S) {
+                w.unit = u;
+                w.slot = rem;
+                w.j0 = (int)((unsigned)rem * (unsigned)nkv / (unsigned)S);
+                w.j1 = (int)((unsigned)(rem + 1) * (unsigned)nkv / (unsigned)S);
                 break;
             }
-            rem -= per_head * a.Hkv;
+            rem -= S;
         }
-        if (b == a.batch) { w.b = -1; w.j0 = w.j1 = 0; w.g = w.unit = w.slot = 0; w.L = w.n = w.row_base = 0; }
     }
     return w;
 }
@@ -291,13 +293,16 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     const uint32_t bar_p_full = bar_s_full + 8 * kScoreBufs;     // (CTA 0) [kScoreBufs] P written by both CTAs
     const uint32_t bar_pv_done = bar_p_full + 8 * kScoreBufs;    // [4] PV of tile j landed: barrier j % 4
     const uint32_t bar_o_full = bar_pv_done + 32;                // last PV landed
-    const uint32_t bar_xch = bar_o_full + 8;                     // [4] the kParts warps of a lane quarter meet here
+    const uint32_t bar_xch = bar_o_full + 8;                     // [4] the warps of a lane quarter meet here (row sums)
     const uint32_t bar_rare = bar_xch + 32;                      // [4] ... and here when a row's reference has to move
-    const uint32_t tmem_slot = bar_rare + 32;                    // uint32
-    static_assert(8 * (1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5 + 8) + 8 <= kSmemBarBytes, "barrier area");
+    const uint32_t bar_ref = bar_rare + 32;                      // [4] the rows' references are published
+    const uint32_t tmem_slot = bar_ref + 32;                     // uint32
+    constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 4 + 1 + 4 + 4 + 4;
+    static_assert(8 * kNumBars + 8 <= kSmemBarBytes, "barrier area");
+    static_assert(kNumBars <= 64, "one thread of warps 2-3 per barrier");
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem_gen + (tmem_slot - smem_base) + 4);
-    float* s_xch = reinterpret_cast<float*>(smem_gen + kSmemXchOff);
+    float* s_xch = reinterpret_cast<float*>(smem_gen + kSmemXchOff);      // [128 rows]: published references
     float* s_cand = reinterpret_cast<float*>(smem_gen + kSmemCandOff);
     volatile int* s_req = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff);        // [4]
     volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff) + 4;    // [4][kParts]
@@ -306,7 +311,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;   // 0: issues the MMAs, owns the "(CTA 0)" barriers
     if (threadIdx.x == 0) EVLN_STAMP(0);
 
-    const WorkItem w = decode_work<PAGED, LensT, kItemRows>(a, lens, CTAS == 2 ? blockIdx.x >> 1 : blockIdx.x);
+    const WorkItem w = decode_work<PAGED, LensT, CTAS>(a, lens);
     if (PAGED && w.b < 0) return;                      // both CTAs of the pair decode the same item
 
     const int rows_valid = w.n * a.G;                            // packed rows of this episode
@@ -336,7 +341,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     }
 
     // ---- setup: barriers, TMEM, then the pair synchronises once ----
-    if (threadIdx.x == 32) {
+    if (threadIdx.x == 0) {
         ptx::prefetch_tensormap(&tm_q);
         ptx::prefetch_tensormap(&tm_k);
         ptx::prefetch_tensormap(&tm_v);
@@ -356,14 +361,14 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     if (warp == 2 || warp == 3) {
         // one barrier per thread: arrival counts in the order of the barrier area
         const int i = (int)threadIdx.x - 64;
-        constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 4 + 1 + 4 + 4;
         if (i < kNumBars) {
             int count = 1;
             if (i < 1 + kKStages + kVStages) count = CTAS;                                // q_full, k_full, v_full
             else if (i < 1 + 2 * kKStages + 2 * kVStages + kScoreBufs) count = 1;         // k_empty, v_empty, s_full
-            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs) count = CTAS * quarters * kParts;   // p_full: every softmax warp
+            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs) count = CTAS * quarters * 2;   // p_full: the tile's softmax warps
             else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5) count = 1;  // pv_done, o_full
-            else count = kParts;                                                          // xch, rare
+            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5 + 8) count = kParts;   // xch, rare
+            else count = 1;                                                               // ref
             ptx::mbar_init(bar_base + 8 * i, count);
             ptx::fence_barrier_init();
         }
@@ -551,17 +556,19 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 ok = __all_sync(0xffffffffu, mine);
             }
             if (!ok) break;
-            if (lane == 0 && jj < 8) EVLN_STAMP(33 + 3 * jj);
+            if (lane == 0 && jj < 12) EVLN_STAMP(20 + jj);
             ptx::fence_after_sync();
             issue_pv(jj);
             if (jn < ntiles) issue_s(jn);
-            if (lane == 0 && jj < 8) EVLN_STAMP(34 + 3 * jj);
+            if (lane == 0 && jj < 12) EVLN_STAMP(32 + jj);
             __syncwarp();
         }
     } else if (warp >= 4 && (warp & 3) < quarters) {
         // ================= softmax + epilogue =================
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
-        const int part = (warp - 4) >> 2;                  // which 32 columns of a row
+        const int part = (warp - 4) >> 2;                  // its 32 channels of O (epilogue, rescales)
+        const int grp = part >> 1;                         // its KV tiles: grp, grp + 2, ...
+        const int half = part & 1;                         // its score columns: [64 half, +64), two blocks of 32
         const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
         const int r_local = row0 + r_tile;                 // packed row within the episode
         const bool row_valid = r_local < rows_valid;
@@ -611,23 +618,37 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             return __shfl_sync(0xffffffffu, r, 0);
         };
 
-        // The exponentials of a row are taken against a reference m_ref that its kParts threads fix
-        // together on the first tile and then leave alone: the division by the row sum at the end
-        // makes any reference exact, and floating point keeps the relative precision as long as
-        // nothing overflows, i.e. as long as no score exceeds the reference by more than
-        // 2^kRefHeadroom.  So after the first tile the warps of a lane quarter do not talk to each
-        // other at all and drift apart, which is what hides their barrier, TMEM and special-function
-        // latencies behind one another.  A thread that does meet such a score asks for a new
-        // reference: every warp of the quarter comes here at its next tile boundary (or out of a
-        // wait), with `released` = the number of tiles whose P it has handed to the tensor core.
-        // Nothing of a tile is consumed before all its parts are handed over, so the slowest warp
+        // The exponentials of a row are taken against a reference m_ref that is fixed once (below) and
+        // then left alone: the division by the row sum at the end makes any reference exact, and
+        // floating point keeps the relative precision as long as nothing overflows, i.e. as long as
+        // no score exceeds the reference by more than 2^kRefHeadroom.  So the warps of a lane quarter
+        // do not talk to each other while they work and drift apart, which is what hides their
+        // barrier, TMEM and special-function latencies behind one another.  A thread that does meet
+        // such a score asks for a new reference: every warp of the quarter comes here at its next
+        // tile boundary (or out of a wait), with `released` = the first tile it has not handed to the
+        // tensor core yet (it has handed over all its tiles below) and `blocks` = how many 32-column
+        // blocks of that tile it has already written.  Nothing of a tile is consumed before all its
+        // parts are handed over and the products are issued in tile order, so the smallest `released`
         // bounds what the accumulator holds; everybody then moves its own state to the new reference
-        // (a power-of-two factor, exact): running sum, its channels of O, and its parts of the P
+        // (a power-of-two factor, exact): running sum, its channels of O, and its blocks of the P
         // tiles that are written but not yet consumed.
         int nrare = 0;                // meetings on bar_rare so far
         bool sum_published = false;   // this thread's share of the row sum is out for the final exchange
         float* s_sum = s_xch + kParts * 128;
-        auto move_reference = [&](int released, bool mine, float want) -> bool {
+        auto scale_p_block = [&](int t, int blk, float alpha) {
+            uint32_t pk[16];
+            const uint32_t t_pt = t_lane + (t % kScoreBufs) * 128 + half * 64 + blk * 32;
+            ptx::tmem_ld16(t_pt, pk);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const float lo = __uint_as_float(pk[e] << 16) * alpha;
+                const float hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
+                pk[e] = ptx::pack_bf16x2(lo, hi);
+            }
+            ptx::tmem_st16(t_pt, pk);
+        };
+        auto move_reference = [&](int released, int blocks, bool mine, float want) -> bool {
             s_cand[part * 128 + r_tile] = mine ? want : m_ref;
             if (lane == 0) s_rel[quarter * kParts + part] = released;
             __syncwarp();
@@ -655,9 +676,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             const bool any_change = __any_sync(0xffffffffu, alpha != 1.f);
             if (any_change) {
                 if (r_min > 0) {
-                    // PV(r_min - 1) must have landed.  The slowest warp saw the scores of tile r_min - 1,
-                    // which were written after PV(r_min - 4): at most three products are outstanding and
-                    // barrier (r_min - 1) % 4 has seen (r_min - 1) / 4 or one more phase.
+                    // PV(r_min - 1) must have landed.  Every tile below r_min is handed over, tile r_min
+                    // is not, and the products are issued in order: PV(r_min + 3) cannot have been
+                    // issued, so barrier (r_min - 1) % 4 has seen (r_min - 1) / 4 phases or one more.
                     if (!warp_wait(bar_pv_done + 8 * ((r_min - 1) & 3), ((r_min - 1) >> 2) & 1, kDevTimeoutSoftmaxO, a.status,
                                    s_abort, lane))
                         return false;
@@ -669,19 +690,14 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                     for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
                     ptx::tmem_st32(t_o, regs);
                 }
-                for (int t = r_min; t < released; ++t) {    // written, not consumed: at most three tiles
-                    uint32_t pk[16];
-                    const uint32_t t_pt = t_lane + (t % kScoreBufs) * 128 + part * 32;
-                    ptx::tmem_ld16(t_pt, pk);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float lo = __uint_as_float(pk[e] << 16) * alpha;
-                        const float hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
-                        pk[e] = ptx::pack_bf16x2(lo, hi);
-                    }
-                    ptx::tmem_st16(t_pt, pk);
+                // written, not consumed: this warp's tiles in [r_min, released) and the blocks of the
+                // tile it is working on
+                for (int t = r_min; t < released; ++t) {
+                    if ((t & 1) != grp) continue;
+                    scale_p_block(t, 0, alpha);
+                    scale_p_block(t, 1, alpha);
                 }
+                for (int blk = 0; blk < blocks; ++blk) scale_p_block(released, blk, alpha);
                 l *= alpha;
                 ptx::tmem_st_wait();
                 ptx::fence_before_sync();
@@ -691,66 +707,81 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             return meet(bar_rare, nrare++);
         };
 
-        for (int jj = 0; jj < ntiles; ++jj) {
+        // The row's reference: the largest of its first 32 scores of the item's first tile (-inf: the
+        // row sees no key of this split, since the visible keys of a row are a prefix).  The thread that
+        // owns those columns reads it off and publishes it; nobody can ask for a new reference before.
+        if (part == 0) {
+            ok = warp_wait(bar_s_full, 0, kDevTimeoutSoftmaxS, a.status, s_abort, lane);
+            if (ok) {
+                ptx::fence_after_sync();
+                uint32_t s0[32];
+                ptx::tmem_ld32(t_lane, s0);
+                ptx::tmem_ld_wait();
+                const int lim = bound - w.j0 * kTileN;
+                if (lim < 31) mask32(s0, lim);
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                rowmax32(s0, mx0, mx1, mx2, mx3);
+                m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
+                s_xch[r_tile] = m_ref;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_ref + 8 * quarter);
+            }
+        } else {
+            ok = warp_wait(bar_ref + 8 * quarter, 0, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
+            if (ok) m_ref = s_xch[r_tile];
+        }
+
+        for (int jj = grp; jj < ntiles && ok; jj += 2) {
             const int buf = jj % kScoreBufs;
             while (ok) {
                 const int r = wait_or_request(bar_s_full + 8 * buf, (jj / kScoreBufs) & 1, kDevTimeoutSoftmaxS);
                 if (r == 0) break;
-                ok = (r == 1) && move_reference(jj, false, 0.f);
+                ok = (r == 1) && move_reference(jj, 0, false, 0.f);
             }
             if (!ok) break;
             ptx::fence_after_sync();
-            if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(2 + 3 * jj);
+            if (half == 0 && quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(2 + jj);
 
-            const int lim = bound - (w.j0 + jj) * kTileN - part * 32;   // columns 0..lim of this part are visible
-            const bool no_mask = __all_sync(0xffffffffu, lim >= 31);
-            const uint32_t t_s = t_lane + buf * 128 + part * 32;
-            const uint32_t t_p = t_s;       // P over this thread's own score columns only: nobody else's are touched
-
-            uint32_t sA[32];
-            ptx::tmem_ld32(t_s, sA);
-            ptx::tmem_ld_wait();
-            if (!no_mask) mask32(sA, lim);  // -inf: masked keys (and stale slots) drop out
-
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-            rowmax32(sA, mx0, mx1, mx2, mx3);
-            float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
-            if (jj == 0) {
-                // the row's reference: its maximum over the whole first tile (-inf: no visible key yet)
-                s_xch[part * 128 + r_tile] = tmax;
-                ok = meet(bar_xch, 0);
-                if (!ok) break;
 #pragma unroll
-                for (int c = 0; c < kParts; ++c) tmax = fmaxf(tmax, s_xch[c * 128 + r_tile]);
-                m_ref = tmax;
-            } else {
+            for (int blk = 0; blk < 2; ++blk) {
+                const int c0 = half * 64 + blk * 32;
+                const int lim = bound - (w.j0 + jj) * kTileN - c0;   // columns 0..lim of this block are visible
+                const bool no_mask = __all_sync(0xffffffffu, lim >= 31);
+                const uint32_t t_s = t_lane + buf * 128 + c0;        // P goes over this thread's own score columns only
+
+                uint32_t sA[32];
+                ptx::tmem_ld32(t_s, sA);
+                ptx::tmem_ld_wait();
+                if (!no_mask) mask32(sA, lim);  // -inf: masked keys (and stale slots) drop out
+
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                rowmax32(sA, mx0, mx1, mx2, mx3);
+                const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
                 bool over = tmax > m_ref + kRefHeadroom;
                 while (ok && __any_sync(0xffffffffu, over)) {
-                    ok = move_reference(jj, over, tmax);
+                    ok = move_reference(jj, blk, over, tmax);
                     over = tmax > m_ref + kRefHeadroom;
                 }
                 if (!ok) break;
-            }
-            if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(3 + 3 * jj);
 
-            // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P over the S columns
-            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
-            uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
-            exp32_store(sA, t_p, scale2, negm2, sum2a, sum2b);
-            {
+                // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P over the S columns
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
+                uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
+                exp32_store(sA, t_s, scale2, negm2, sum2a, sum2b);
                 float a0, a1, b0, b1;
                 ptx::unpack2(sum2a, a0, a1);
                 ptx::unpack2(sum2b, b0, b1);
                 l += (a0 + a1) + (b0 + b1);
             }
+            if (!ok) break;
             ptx::tmem_st_wait();
             ptx::fence_before_sync();
             __syncwarp();
             if (lane == 0) {
                 if (CTAS == 2) ptx::mbar_arrive_cluster(p_full0 + 8 * buf); else ptx::mbar_arrive(p_full0 + 8 * buf);
             }
-            if (warp == 4 && lane == 0 && jj < 10) EVLN_STAMP(4 + 3 * jj);
+            if (half == 0 && quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(11 + jj);
         }
 
         // All tiles handed over.  The row sum is the sum over the row's threads (same reference in
@@ -764,9 +795,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
         }
         while (ok) {
-            const int r = wait_or_request(bar_xch + 8 * quarter, 1, kDevTimeoutSoftmaxX);
+            const int r = wait_or_request(bar_xch + 8 * quarter, 0, kDevTimeoutSoftmaxX);
             if (r == 0) break;
-            ok = (r == 1) && move_reference(ntiles, false, 0.f);
+            ok = (r == 1) && move_reference(ntiles, 0, false, 0.f);
         }
         // nobody of the quarter can ask any more; the last product
         if (ok) ok = warp_wait(bar_o_full, 0, kDevTimeoutSoftmaxO, a.status, s_abort, lane);

@@ -30,6 +30,7 @@ enum DeviceStatus : int {
 struct BatchLens {
     int cache_len[kMaxBatch];
     int new_off[kMaxBatch + 1];
+    int item_off[kMaxBatch + 1];   // first work item of the attention kernel per episode
 };
 
 template <typename T> struct VecTraits;
@@ -54,10 +55,40 @@ __host__ __device__ inline int unit_kv_tiles(int L, int n, int G, int unit, int 
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Division of x < 2^31 by a constant d >= 1 as a multiplication: with l = ceil(log2 d) and
+// mul = ceil(2^(31+l) / d) < 2^32, floor(x * mul / 2^(31+l)) = floor(x / d) exactly (the error
+// x * (mul*d - 2^(31+l)) / (d * 2^(31+l)) stays below 2^-l <= 1/d).  An integer division costs a
+// CTA a few hundred cycles of latency before it knows what to load.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+inline FastDiv make_fast_div(uint32_t d)
+{
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    FastDiv f;
+    f.shift = 31 + l;
+    f.mul = (uint32_t)(((1ull << f.shift) + d - 1) / d);
+    return f;
+}
+__host__ __device__ inline uint32_t fast_div(uint32_t x, FastDiv f)
+{
+    return (uint32_t)(((unsigned long long)x * f.mul) >> f.shift);
+}
+// unit_kv_tiles with the division by G prepared by the host
+__host__ __device__ inline int unit_kv_tiles_fast(int L, int n, FastDiv div_g, int unit, int unit_rows)
+{
+    const uint32_t last_row = (uint32_t)(unit + 1) * (uint32_t)unit_rows - 1u;
+    uint32_t last_tok = fast_div(last_row, div_g);
+    if (last_tok > (uint32_t)(n - 1)) last_tok = (uint32_t)(n - 1);
+    return (int)(((uint32_t)L + last_tok + 1u + (uint32_t)kTileN - 1u) / (uint32_t)kTileN);
+}
+
 // Stub lengths for the kernels that serve one episode.
 struct NoLens {
     int cache_len[1];
     int new_off[2];
+    int item_off[2];
 };
 
 }  // namespace evln

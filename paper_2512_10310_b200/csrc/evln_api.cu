@@ -34,8 +34,12 @@ struct evlnContext {
 };
 
 #ifdef EVLN_TIMELINE
-static long long* g_timeline = nullptr;
-extern "C" void evlnDebugSetTimeline(void* p) { g_timeline = (long long*)p; }
+// debug builds only (see timeline_debug.cuh): where the attention kernel leaves its clock stamps
+extern "C" int evlnDebugSetTimeline(void* p)
+{
+    long long* v = (long long*)p;
+    return (int)cudaMemcpyToSymbol(evln::g_timeline_dev, &v, sizeof(v));
+}
 #endif
 
 namespace {
@@ -62,10 +66,10 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 // The attention kernel runs as clusters of two CTAs (one CTA pair per work item).
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pair_pdl(void (*kernel)(KArgs...), int items, size_t smem, cudaStream_t st, Args&&... args)
+cudaError_t launch_pair_pdl(void (*kernel)(KArgs...), dim3 grid, size_t smem, cudaStream_t st, Args&&... args)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * items);
+    cfg.gridDim = grid;                 // x: two CTAs per work item
     cfg.blockDim = dim3(kTcThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -251,11 +255,26 @@ void paged_schedule(evlnHandle_t h, const evlnPagedParams* p, const int* lens, c
     *items = cnt * p->num_kv_heads;
 }
 
-void fill_lens(BatchLens* bl, const evlnPagedParams* p, const int* lens, const int* offs)
+// chunk_tiles > 0: also the first attention work item of every episode (items are numbered
+// episode by episode: kv head, unit, split)
+void fill_lens(BatchLens* bl, const evlnPagedParams* p, const int* lens, const int* offs, int chunk_tiles = 0)
 {
     memset(bl, 0, sizeof(*bl));
     for (int b = 0; b < p->batch; ++b) bl->cache_len[b] = lens[b];
     for (int b = 0; b <= p->batch; ++b) bl->new_off[b] = offs[b];
+    if (chunk_tiles > 0) {
+        const int G = p->num_q_heads / p->num_kv_heads;
+        int items = 0;
+        for (int b = 0; b < p->batch; ++b) {
+            bl->item_off[b] = items;
+            const int n = offs[b + 1] - offs[b];
+            const int units = ceil_div(n * G, kUnitRows);
+            int per_head = 0;
+            for (int u = 0; u < units; ++u) per_head += ceil_div(unit_kv_tiles(lens[b], n, G, u, kUnitRows), chunk_tiles);
+            items += per_head * p->num_kv_heads;
+        }
+        for (int b = p->batch; b <= kMaxBatch; ++b) bl->item_off[b] = items;
+    }
 }
 
 template <typename T>
@@ -465,15 +484,16 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
         a.cache_len = p->cache_len; a.num_new = p->num_new; a.num_splits = S;
         a.units_per_head = use_solo_kernel(p) ? 1 : ceil_div(R, kUnitRows);
         a.scale_log2 = scale * 1.4426950408889634f;
-#ifdef EVLN_TIMELINE
-        a.timeline = g_timeline;
-#endif
+        a.div_g = make_fast_div((uint32_t)G);
+        a.div_s = make_fast_div((uint32_t)S);
         NoLens nl = {};
-        const int items = S * p->num_kv_heads * a.units_per_head;
+        // one work item per (unit, kv head, split): the kernels read it off the block index
+        if (a.units_per_head > 32767 || p->num_kv_heads > 65535) return EVLN_NOT_SUPPORTED;
         if (use_solo_kernel(p))
-            launch_pdl(attn_solo_kernel, dim3(items), dim3(kTcThreads), kSoloSmemBytes, st, tm_q, tm_k, tm_v, a);
+            launch_pdl(attn_solo_kernel, dim3(1, p->num_kv_heads, S), dim3(kTcThreads), kSoloSmemBytes, st, tm_q, tm_k, tm_v, a);
         else
-            launch_pair_pdl(attn_pair_kernel<false, NoLens>, items, kTcSmemBytes, st, tm_q, tm_k, tm_v, a, nl);
+            launch_pair_pdl(attn_pair_kernel<false, NoLens>, dim3(2 * a.units_per_head, p->num_kv_heads, S), kTcSmemBytes, st,
+                            tm_q, tm_k, tm_v, a, nl);
     } else {
         SimtAttnArgs a = {};
         a.q_rot = q_rot; a.k_cache = k_cache; a.v_cache = v_cache;
@@ -621,9 +641,13 @@ evlnStatus_t evlnPagedStepAttention(evlnHandle_t h, const evlnPagedParams* p, co
     a.Hkv = p->num_kv_heads; a.G = G; a.rows = (int)rows;
     a.batch = p->batch; a.max_pages = p->max_pages_per_seq; a.chunk_tiles = chunk;
     a.scale_log2 = scale * 1.4426950408889634f;
+    a.div_g = make_fast_div((uint32_t)G);
+    a.div_s = make_fast_div(1u);
     BatchLens bl;
-    fill_lens(&bl, p, h_cache_lens, h_new_offsets);
-    launch_pair_pdl(attn_pair_kernel<true, BatchLens>, (int)items, kTcSmemBytes, (cudaStream_t)stream, tm_q, tm_k, tm_v, a, bl);
+    fill_lens(&bl, p, h_cache_lens, h_new_offsets, chunk);
+    if (bl.item_off[p->batch] != (int)items) return EVLN_INVALID_VALUE;
+    launch_pair_pdl(attn_pair_kernel<true, BatchLens>, dim3(2 * (int)items), kTcSmemBytes, (cudaStream_t)stream, tm_q, tm_k,
+                    tm_v, a, bl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
