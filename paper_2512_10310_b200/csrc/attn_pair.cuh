@@ -12,31 +12,31 @@
 // query rows.  The item's normalised partial outputs + log-sum-exps go to the workspace that
 // the combine kernel merges.
 //
-// Per CTA (640 threads, 1 CTA/SM, ~199 KB shared memory, all 512 TMEM columns):
+// Per CTA (384 threads, 1 CTA/SM, ~199 KB shared memory, all 512 TMEM columns):
 //   warp 0      TMA producer: the CTA's Q tile once, then its K / V half tiles through two
 //               5-deep rings of 16 KB stages (128B-swizzled); no multicast anywhere.  Bytes are
-//               counted on barriers of CTA 0, where the MMA thread waits.
-//   warp 1      (CTA 0) MMA issuer, one elected lane: S_j = Q K_j^T (SS) into one of THREE score
-//               buffers, O += P_j V_j (A = P from TMEM).  Scores run up to three tiles ahead
-//               of the softmax, so the tensor pipe and the softmax warps only meet through
-//               full/empty barriers and neither waits for the other's latency.
-//   warps 4-19  softmax + epilogue, four warps per TMEM lane quarter (= per SM sub-partition).
-//               They work in two groups on ALTERNATE KV tiles: the warps of group 0 take the
-//               even tiles of the item, those of group 1 the odd ones, and within a group a
-//               thread owns 64 of the 128 score columns of its row (two blocks of 32).  The two
-//               groups of a sub-partition are therefore half a tile period apart: while one waits
-//               for scores, reads tensor memory or hands over P, the other keeps the 4 SFU lanes
-//               busy with exponentials (a tile's 128x128 exponentials take as long as its MMAs,
-//               so that unit must not idle).  The exponentials of a row are taken against a
-//               reference that one thread of the row reads off the first 32 scores of the first
-//               tile and passes to the other three through shared memory; the threads talk to each
-//               other again only if a later score exceeds it by more than 2^64 (then O, the row
-//               sums and the pending P tiles are rescaled by a power of two); the final division
-//               by the row sum makes any reference exact.  P is written back over the scores as
-//               packed bf16.
-//   warps 2-3   set up the barriers, then idle.
-// TMEM columns: S_b at 128*b, b = 0..2; P_b (packed bf16) sits in columns [32c, 32c+16), c = 0..3,
-// of S_b, each block over the score columns of the thread that writes it; O at 384.
+//               counted on barriers of CTA 0, where the MMA threads wait.
+//   warp 1      (CTA 0) score issuer, one elected lane: S_j = Q K_j^T (SS) into score buffer
+//               j % 2 as soon as the softmax has READ tile j-2 out of it.
+//   warp 2      (CTA 0) product issuer: O += P_j V_j (A = P_j from tensor memory, buffer j % 2)
+//               as soon as P_j is written.  Scores and products have buffers of their own, so
+//               neither instruction stream waits for the other.
+//   warps 4-11  softmax + epilogue, two warps per TMEM lane quarter (= per SM sub-partition), one
+//               thread per query row.  The warps of group 0 take the even KV tiles of the item,
+//               those of group 1 the odd ones: a thread pulls the 128 scores of its row into
+//               registers, gives the score buffer back at once, and then works through its 128
+//               exponentials while the other warp of the sub-partition is in another phase of
+//               another tile (a tile's exponentials keep the 4 SFU lanes of a sub-partition busy
+//               for as long as its MMAs keep the tensor pipe busy, so that unit must not idle).
+//               The exponentials of a row are taken against a reference that the group-0 thread
+//               reads off the first 32 scores of the first tile and passes to the other thread
+//               through shared memory; the two talk to each other again only if a later score
+//               exceeds it by more than 2^64 (then O, the row sums and the pending P tiles are
+//               rescaled by a power of two); the final division by the row sum makes any
+//               reference exact.
+//   warp 3      sets up barriers (with warp 2), then idles.
+// TMEM columns: scores S_b at 128 b, b = 0..1; P_b (128 keys as 64 columns of packed bf16 pairs) at
+// 256 + 64 b; O at 384.
 //
 // Every mbarrier wait is bounded: on expiry the CTA records a code in the device status word and
 // raises a shared abort flag; all roles then leave their loops, TMEM is freed and the pair
@@ -51,12 +51,12 @@
 
 namespace evln {
 
-constexpr int kTcThreads = 640;
-constexpr int kParts = 4;                             // threads per score row (32 columns each)
+constexpr int kTcThreads = 384;
+constexpr int kGroups = 2;                            // softmax threads per query row: one per tile parity
 constexpr int kTileBytes = kTileM * 128 * 2;          // Q tile: 128 rows x 128 channels x bf16
 constexpr int kHalfBytes = kTileBytes / 2;            // 16 KB: a 64-channel half of Q; a K or V half tile
 constexpr int kSmemBarBytes = 384;
-constexpr int kSmemXchBytes = 2 * kParts * 128 * 4 + kParts * 128 * 4 + 128;
+constexpr int kSmemXchBytes = 128 * 4 + 2 * kGroups * 128 * 4 + 128;
 
 // Shared-memory plan of a CTA.  CTAS = 2: the CTA of a pair stages half tiles (16 KB) through two
 // 5-deep rings.  CTAS = 1: a CTA on its own stages whole K / V tiles (32 KB: two 64-channel blocks
@@ -70,17 +70,20 @@ struct SmemPlan {
     static constexpr int kKOff = kTileBytes;
     static constexpr int kVOff = kKOff + kKStages * kStageBytes;
     static constexpr int kBarOff = kVOff + kVStages * kStageBytes;
-    static constexpr int kXchOff = kBarOff + kSmemBarBytes;          // float [2 meetings][kParts][128 rows]
-    static constexpr int kCandOff = kXchOff + 2 * kParts * 128 * 4;  // float [kParts][128 rows]: reference requests
-    static constexpr int kReqOff = kCandOff + kParts * 128 * 4;      // int [4] request flags, int [4][kParts] released tiles
-    static constexpr int kBytes = kXchOff + kSmemXchBytes + 1024;    // + slack to align to 1024
-    static_assert(kKStages * kStageBytes >= 16 * 32 * 144, "the epilogue stages its rows in the K ring");
+    static constexpr int kRefOff = kBarOff + kSmemBarBytes;          // float [128 rows]: published references
+    static constexpr int kSumOff = kRefOff + 128 * 4;                // float [kGroups][128 rows]: row-sum shares
+    static constexpr int kCandOff = kSumOff + kGroups * 128 * 4;     // float [kGroups][128 rows]: reference requests
+    static constexpr int kReqOff = kCandOff + kGroups * 128 * 4;     // int [4] request flags, int [4][kGroups] released tiles
+    static constexpr int kBytes = kRefOff + kSmemXchBytes + 1024;    // + slack to align to 1024
+    static_assert(kKStages * kStageBytes >= 8 * 32 * 144, "the epilogue stages its rows in the K ring");
     static_assert(kBytes <= 227 * 1024, "shared memory per CTA");
 };
 constexpr int kTcSmemBytes = SmemPlan<2>::kBytes;
 constexpr int kSoloSmemBytes = SmemPlan<1>::kBytes;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at boost clocks
-constexpr int kScoreBufs = 3;
+constexpr int kScoreBufs = 2;
+constexpr int kRegsIssue = 80, kRegsSoftmax = 208;    // per thread, after the set-up (4 + 8 warps: 62 K of 64 K registers)
+constexpr uint32_t kColP = 256;
 constexpr uint32_t kColO = 384;
 #ifndef EVLN_REF_HEADROOM
 #define EVLN_REF_HEADROOM 64.f
@@ -156,16 +159,16 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, int cod
     return __shfl_sync(0xffffffffu, r, 0) != 0;
 }
 
-// --- softmax pieces on one 32-column register block of a score row ---------------------------
+// --- softmax pieces on 32-column register blocks of a score row ------------------------------
 
-__device__ __forceinline__ void mask32(uint32_t (&s)[32], int lim)
+__device__ __forceinline__ void mask32(uint32_t* s, int lim)
 {
 #pragma unroll
     for (int e = 0; e < 32; ++e)
         if (e > lim) s[e] = 0xff800000u;
 }
 
-__device__ __forceinline__ void rowmax32(const uint32_t (&s)[32], float& m0, float& m1, float& m2, float& m3)
+__device__ __forceinline__ void rowmax32(const uint32_t* s, float& m0, float& m1, float& m2, float& m3)
 {
 #pragma unroll
     for (int e = 0; e < 32; e += 8) {
@@ -176,12 +179,11 @@ __device__ __forceinline__ void rowmax32(const uint32_t (&s)[32], float& m0, flo
     }
 }
 
-// p = 2^(s*scale + negm) for 32 columns, accumulated into two packed sums, written to TMEM as
-// 16 columns of packed bf16 pairs
-__device__ __forceinline__ void exp32_store(const uint32_t (&s)[32], uint32_t taddr, uint64_t scale2,
-                                            uint64_t negm2, uint64_t& sum2a, uint64_t& sum2b)
+// p = 2^(s*scale + negm) for 32 columns, accumulated into two packed sums, left as 16 packed
+// bf16 pairs (= 16 columns of tensor memory)
+__device__ __forceinline__ void exp32(const uint32_t* s, uint32_t (&packed)[16], uint64_t scale2,
+                                      uint64_t negm2, uint64_t& sum2a, uint64_t& sum2b)
 {
-    uint32_t packed[16];
 #pragma unroll
     for (int e = 0; e < 32; e += 4) {
         const uint64_t xa = ptx::fma2(ptx::pack2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), scale2, negm2);
@@ -195,7 +197,6 @@ __device__ __forceinline__ void exp32_store(const uint32_t (&s)[32], uint32_t ta
         packed[e >> 1] = ptx::pack_bf16x2(p0, p1);
         packed[(e >> 1) + 1] = ptx::pack_bf16x2(p2, p3);
     }
-    ptx::tmem_st16(taddr, packed);
 }
 
 // --- work decoding ------------------------------------------------------------------------
@@ -264,8 +265,8 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
 }
 
 // --- the kernel ---------------------------------------------------------------------------
-// CTAS = 2: launched with a cluster of 2 CTAs along x: work item = blockIdx.x / 2, query tile = rank.
-// CTAS = 1: no cluster; work item = blockIdx.x, one query tile (all the rows of a kv head fit in it).
+// CTAS = 2: launched with a cluster of 2 CTAs along x: query tile = cluster rank.
+// CTAS = 1: no cluster; one query tile (all the rows of a kv head fit in it).
 
 template <bool PAGED, typename LensT, int CTAS>
 __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
@@ -275,37 +276,40 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     using Plan = SmemPlan<CTAS>;
     constexpr int kKStages = Plan::kKStages, kVStages = Plan::kVStages, kStageBytes = Plan::kStageBytes;
     constexpr int kSmemQOff = Plan::kQOff, kSmemKOff = Plan::kKOff, kSmemVOff = Plan::kVOff;
-    constexpr int kSmemBarOff = Plan::kBarOff, kSmemXchOff = Plan::kXchOff, kSmemCandOff = Plan::kCandOff;
-    constexpr int kSmemReqOff = Plan::kReqOff;
     constexpr int kItemRows = CTAS * kTileM;           // query rows of a work item
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
 
     // barriers: same offsets in both CTAs; "(CTA 0)" marks those of which only CTA 0's copy is used
-    const uint32_t bar_base = smem_base + kSmemBarOff;
+    const uint32_t bar_base = smem_base + Plan::kBarOff;
     const uint32_t bar_q_full = bar_base;                        // (CTA 0) both CTAs' Q tiles landed
     const uint32_t bar_k_full = bar_q_full + 8;                  // (CTA 0) [kKStages]
     const uint32_t bar_v_full = bar_k_full + 8 * kKStages;       // (CTA 0) [kVStages]
-    const uint32_t bar_k_empty = bar_v_full + 8 * kVStages;      // [kKStages] stage consumed by the MMAs
+    const uint32_t bar_s_free = bar_v_full + 8 * kVStages;       // (CTA 0) [kScoreBufs] scores read by both CTAs' softmax
+    const uint32_t bar_p_full = bar_s_free + 8 * kScoreBufs;     // (CTA 0) [kScoreBufs] P written by both CTAs
+    const uint32_t bar_k_empty = bar_p_full + 8 * kScoreBufs;    // [kKStages] stage consumed by the MMAs
     const uint32_t bar_v_empty = bar_k_empty + 8 * kKStages;     // [kVStages]
     const uint32_t bar_s_full = bar_v_empty + 8 * kVStages;      // [kScoreBufs] scores ready
-    const uint32_t bar_p_full = bar_s_full + 8 * kScoreBufs;     // (CTA 0) [kScoreBufs] P written by both CTAs
-    const uint32_t bar_pv_done = bar_p_full + 8 * kScoreBufs;    // [4] PV of tile j landed: barrier j % 4
+    const uint32_t bar_pv_done = bar_s_full + 8 * kScoreBufs;    // [4] PV of tile j landed: barrier j % 4
     const uint32_t bar_o_full = bar_pv_done + 32;                // last PV landed
-    const uint32_t bar_xch = bar_o_full + 8;                     // [4] the warps of a lane quarter meet here (row sums)
+    const uint32_t bar_ref = bar_o_full + 8;                     // [4] the rows' references are published
+    const uint32_t bar_xch = bar_ref + 32;                       // [4] the two warps of a lane quarter meet here (row sums)
     const uint32_t bar_rare = bar_xch + 32;                      // [4] ... and here when a row's reference has to move
-    const uint32_t bar_ref = bar_rare + 32;                      // [4] the rows' references are published
-    const uint32_t tmem_slot = bar_ref + 32;                     // uint32
-    constexpr int kNumBars = 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 4 + 1 + 4 + 4 + 4;
+    const uint32_t tmem_slot = bar_rare + 32;                    // uint32
+    constexpr int kBarsCtas = 1 + kKStages + kVStages;                                 // arrival count CTAS
+    constexpr int kBarsSoft = 2 * kScoreBufs;                                          // one per softmax warp of the tile
+    constexpr int kBarsOne = kKStages + kVStages + kScoreBufs + 4 + 1 + 4;             // count 1
+    constexpr int kNumBars = kBarsCtas + kBarsSoft + kBarsOne + 8;                     // + xch, rare: kGroups
     static_assert(8 * kNumBars + 8 <= kSmemBarBytes, "barrier area");
     static_assert(kNumBars <= 64, "one thread of warps 2-3 per barrier");
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem_gen + (tmem_slot - smem_base) + 4);
-    float* s_xch = reinterpret_cast<float*>(smem_gen + kSmemXchOff);      // [128 rows]: published references
-    float* s_cand = reinterpret_cast<float*>(smem_gen + kSmemCandOff);
-    volatile int* s_req = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff);        // [4]
-    volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + kSmemReqOff) + 4;    // [4][kParts]
+    float* s_ref = reinterpret_cast<float*>(smem_gen + Plan::kRefOff);
+    float* s_sum = reinterpret_cast<float*>(smem_gen + Plan::kSumOff);
+    float* s_cand = reinterpret_cast<float*>(smem_gen + Plan::kCandOff);
+    volatile int* s_req = reinterpret_cast<volatile int*>(smem_gen + Plan::kReqOff);        // [4]
+    volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + Plan::kReqOff) + 4;    // [4][kGroups]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;   // 0: issues the MMAs, owns the "(CTA 0)" barriers
@@ -348,7 +352,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         if (!PAGED) {
             // this CTA's halves of the first K tiles and of the first V tile on their way into L2 while
             // the pair sets up (cached rows; a row the previous kernel is still writing stays coherent)
-            const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
+            const int pre = ntiles < 3 ? ntiles : 3;
             for (int jj = 0; jj < pre; ++jj) {
                 const int key0 = (w.j0 + jj) * kTileN + (int)rank * 64;
                 ptx::tma_prefetch_3d(&tm_k, 0, key0, w.g);
@@ -363,12 +367,10 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         const int i = (int)threadIdx.x - 64;
         if (i < kNumBars) {
             int count = 1;
-            if (i < 1 + kKStages + kVStages) count = CTAS;                                // q_full, k_full, v_full
-            else if (i < 1 + 2 * kKStages + 2 * kVStages + kScoreBufs) count = 1;         // k_empty, v_empty, s_full
-            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs) count = CTAS * quarters * 2;   // p_full: the tile's softmax warps
-            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5) count = 1;  // pv_done, o_full
-            else if (i < 1 + 2 * kKStages + 2 * kVStages + 2 * kScoreBufs + 5 + 8) count = kParts;   // xch, rare
-            else count = 1;                                                               // ref
+            if (i < kBarsCtas) count = CTAS;                                   // q_full, k_full, v_full
+            else if (i < kBarsCtas + kBarsSoft) count = CTAS * quarters;       // s_free, p_full: the tile's softmax warps
+            else if (i < kBarsCtas + kBarsSoft + kBarsOne) count = 1;          // k_empty .. ref
+            else count = kGroups;                                              // xch, rare
             ptx::mbar_init(bar_base + 8 * i, count);
             ptx::fence_barrier_init();
         }
@@ -397,6 +399,12 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     ptx::grid_launch_dependents();
     if (threadIdx.x == 0) EVLN_STAMP(1);
 
+    auto on_cta0 = [&](uint32_t bar) -> uint32_t { return CTAS == 2 ? ptx::map_to_cta(bar, 0) : bar; };
+
+    // Registers go where the work is: the warpgroup of the producer and the issuers gives most of its
+    // share back, the two softmax warpgroups (128 scores per thread in flight) take it.
+    if (warp < 4) {
+    ptx::setmaxnreg_dec<kRegsIssue>();
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
@@ -409,7 +417,6 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             auto tma3 = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
                 if (CTAS == 2) ptx::tma_load_3d_pair(dst, map, bar, x, y, z); else ptx::tma_load_3d(dst, map, bar, x, y, z);
             };
-            auto on_cta0 = [&](uint32_t bar) -> uint32_t { return CTAS == 2 ? ptx::map_to_cta(bar, 0) : bar; };
             {
                 const uint32_t q_full0 = on_cta0(bar_q_full);
                 const uint32_t dst = smem_base + kSmemQOff;
@@ -467,7 +474,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                     ptx::tma_load_4d_pair(dst + 8192, &tm_v, bar, 64 * (int)rank, 0, w.g, pt[p1]);
                 }
             };
-            // in the order the MMAs consume them: K_0..K_2, then V_j, K_{j+3}
+            // in the order the MMAs consume them: K_0, K_1, then V_j, K_{j+2}
             const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
             for (int jj = 0; jj < pre && ok; ++jj) load_k(jj);
             for (int jj = 0; jj < ntiles && ok; ++jj) {
@@ -482,118 +489,125 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         }
         __syncwarp();
     } else if (warp == 1 && rank == 0) {
-        // ================= MMA issuer (CTA 0 of the pair) =================
+        // ================= score issuer (CTA 0 of the pair): S_jj = Q K_jj^T =================
         const uint32_t idesc_s = make_idesc(false, CTAS * kTileM, kTileN);
-        const uint32_t idesc_pv = make_idesc(true, CTAS * kTileM, 128);
-        auto mma_ss = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t idesc, bool acc) {
-            if (CTAS == 2) ptx::mma_ss_pair(d, ad, bd, idesc, acc); else ptx::mma_ss(d, ad, bd, idesc, acc);
-        };
-        auto mma_ts = [&](uint32_t d, uint32_t at, uint64_t bd, uint32_t idesc, bool acc) {
-            if (CTAS == 2) ptx::mma_ts_pair(d, at, bd, idesc, acc); else ptx::mma_ts(d, at, bd, idesc, acc);
-        };
-        auto commit = [&](uint32_t bar) {      // the barrier of that name in every CTA of the item
-            if (CTAS == 2) ptx::mma_commit_pair(bar, (uint16_t)3); else ptx::mma_commit(bar);
-        };
-        bool ok = true;
-        auto wait_u = [&](uint32_t bar, uint32_t parity, int code) -> bool {
-            return warp_wait(bar, parity, code, a.status, s_abort, lane);
-        };
         // descriptors differ only in their address field (units of 16 bytes): build them once
         const uint64_t qdesc0 = make_sdesc(smem_base + kSmemQOff, 16, 1024);
         const uint64_t kdesc0 = make_sdesc(smem_base + kSmemKOff, 16, 1024);            // K-major; 64 (pair) or 128 keys per CTA
-        const uint64_t vdesc0 = make_sdesc(smem_base + kSmemVOff, kHalfBytes, 1024);    // MN-major; 64-channel blocks 16 KB apart
-        auto issue_s = [&](int jj) {             // S_jj = Q K_jj^T into score buffer jj % 3
+        bool ok = warp_wait(bar_q_full, 0, kDevTimeoutMmaQ, a.status, s_abort, lane);
+        for (int jj = 0; jj < ntiles && ok; ++jj) {
+            // K_jj landed; the softmax has read tile jj - 2 out of this score buffer.  A wait costs
+            // ~150 cycles even on a completed barrier, so two lanes take one each.
+            {
+                uint32_t bar = bar_k_full + 8 * (jj % kKStages), parity = (jj / kKStages) & 1;
+                int code = kDevTimeoutMmaKV;
+                if (lane == 1) { bar = bar_s_free + 8 * (jj & 1); parity = ((jj >> 1) - 1) & 1; code = kDevTimeoutMmaP; }
+                bool mine = true;
+                if (lane == 0 || (lane == 1 && jj >= kScoreBufs)) mine = wait_bounded(bar, parity, code, a.status, s_abort);
+                if (lane < 2 && jj < 9) EVLN_STAMP(20 + 9 * lane + jj);
+                ok = __all_sync(0xffffffffu, mine);
+            }
+            if (!ok) break;
+            ptx::fence_after_sync();
             if (ptx::elect_one()) {
                 const int stage = jj % kKStages;
                 const uint64_t kd = kdesc0 + (uint64_t)((stage * kStageBytes) >> 4);
-                const uint32_t d = tmem + (uint32_t)(jj % kScoreBufs) * 128;
+                const uint32_t d = tmem + (uint32_t)(jj & 1) * 128;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t qoff = (uint64_t)(((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4);
                     const uint64_t koff = (uint64_t)(((ks >> 2) * (kStageBytes / 2) + (ks & 3) * 32) >> 4);
-                    mma_ss(d, qdesc0 + qoff, kd + koff, idesc_s, ks > 0);
+                    if (CTAS == 2) ptx::mma_ss_pair(d, qdesc0 + qoff, kd + koff, idesc_s, ks > 0);
+                    else ptx::mma_ss(d, qdesc0 + qoff, kd + koff, idesc_s, ks > 0);
                 }
-                commit(bar_s_full + 8 * (jj % kScoreBufs));
-                commit(bar_k_empty + 8 * stage);
+                if (CTAS == 2) {
+                    ptx::mma_commit_pair(bar_s_full + 8 * (jj & 1), (uint16_t)3);
+                    ptx::mma_commit_pair(bar_k_empty + 8 * stage, (uint16_t)3);
+                } else {
+                    ptx::mma_commit(bar_s_full + 8 * (jj & 1));
+                    ptx::mma_commit(bar_k_empty + 8 * stage);
+                }
             }
-        };
-        auto issue_pv = [&](int jj) {            // O (+)= P_jj V_jj
-            if (ptx::elect_one()) {
-                const int stage = jj % kVStages;
-                const uint64_t vd = vdesc0 + (uint64_t)((stage * kStageBytes) >> 4);
-                const uint32_t p = tmem + (uint32_t)(jj % kScoreBufs) * 128;
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ts(tmem + kColO, p + (ks >> 1) * 32 + (ks & 1) * 8, vd + (uint64_t)((ks * 2048) >> 4),
-                           idesc_pv, jj > 0 || ks > 0);
-                commit(bar_pv_done + 8 * (jj & 3));
-                commit(bar_v_empty + 8 * stage);
-                if (jj == ntiles - 1) commit(bar_o_full);
-            }
-        };
-
-        ok = wait_u(bar_q_full, 0, kDevTimeoutMmaQ);
-        const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
-        for (int jj = 0; jj < pre && ok; ++jj) {
-            ok = wait_u(bar_k_full + 8 * (jj % kKStages), (jj / kKStages) & 1, kDevTimeoutMmaKV);
-            if (ok) {
-                ptx::fence_after_sync();
-                issue_s(jj);
-                __syncwarp();
-            }
+            if (lane == 0 && jj < 9) EVLN_STAMP(38 + jj);
+            __syncwarp();
         }
+    } else if (warp == 2 && rank == 0) {
+        // ================= product issuer (CTA 0 of the pair): O (+)= P_jj V_jj =================
+        const uint32_t idesc_pv = make_idesc(true, CTAS * kTileM, 128);
+        const uint64_t vdesc0 = make_sdesc(smem_base + kSmemVOff, kHalfBytes, 1024);    // MN-major; 64-channel blocks 16 KB apart
+        bool ok = true;
         for (int jj = 0; jj < ntiles && ok; ++jj) {
-            // V_jj, P_jj and K_{jj+3}: a wait costs ~150 cycles even on a completed barrier, so three
-            // lanes take one each and the latencies overlap
-            const int jn = jj + kScoreBufs;
             {
                 uint32_t bar = bar_v_full + 8 * (jj % kVStages), parity = (jj / kVStages) & 1;
                 int code = kDevTimeoutMmaKV;
-                if (lane == 1) { bar = bar_p_full + 8 * (jj % kScoreBufs); parity = (jj / kScoreBufs) & 1; code = kDevTimeoutMmaP; }
-                if (lane == 2) { bar = bar_k_full + 8 * (jn % kKStages); parity = (jn / kKStages) & 1; }
+                if (lane == 1) { bar = bar_p_full + 8 * (jj & 1); parity = (jj >> 1) & 1; code = kDevTimeoutMmaP; }
                 bool mine = true;
-                if (lane < 2 || (lane == 2 && jn < ntiles)) mine = wait_bounded(bar, parity, code, a.status, s_abort);
+                if (lane < 2) mine = wait_bounded(bar, parity, code, a.status, s_abort);
                 ok = __all_sync(0xffffffffu, mine);
             }
             if (!ok) break;
-            if (lane == 0 && jj < 12) EVLN_STAMP(20 + jj);
+            if (lane == 0 && jj < 9) EVLN_STAMP(47 + jj);
             ptx::fence_after_sync();
-            issue_pv(jj);
-            if (jn < ntiles) issue_s(jn);
-            if (lane == 0 && jj < 12) EVLN_STAMP(32 + jj);
+            if (ptx::elect_one()) {
+                const int stage = jj % kVStages;
+                const uint64_t vd = vdesc0 + (uint64_t)((stage * kStageBytes) >> 4);
+                const uint32_t p = tmem + kColP + (uint32_t)(jj & 1) * 64;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    if (CTAS == 2) ptx::mma_ts_pair(tmem + kColO, p + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, jj > 0 || ks > 0);
+                    else ptx::mma_ts(tmem + kColO, p + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), idesc_pv, jj > 0 || ks > 0);
+                }
+                if (CTAS == 2) {
+                    ptx::mma_commit_pair(bar_pv_done + 8 * (jj & 3), (uint16_t)3);
+                    ptx::mma_commit_pair(bar_v_empty + 8 * stage, (uint16_t)3);
+                    if (jj == ntiles - 1) ptx::mma_commit_pair(bar_o_full, (uint16_t)3);
+                } else {
+                    ptx::mma_commit(bar_pv_done + 8 * (jj & 3));
+                    ptx::mma_commit(bar_v_empty + 8 * stage);
+                    if (jj == ntiles - 1) ptx::mma_commit(bar_o_full);
+                }
+            }
             __syncwarp();
         }
-    } else if (warp >= 4 && (warp & 3) < quarters) {
+    }
+    } else {
+    ptx::setmaxnreg_inc<kRegsSoftmax>();
+    if ((warp & 3) < quarters) {
         // ================= softmax + epilogue =================
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
-        const int part = (warp - 4) >> 2;                  // its 32 channels of O (epilogue, rescales)
-        const int grp = part >> 1;                         // its KV tiles: grp, grp + 2, ...
-        const int half = part & 1;                         // its score columns: [64 half, +64), two blocks of 32
+        const int grp = (warp - 4) >> 2;                   // its KV tiles: grp, grp + 2, ...; its 64 channels of O
         const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
         const int r_local = row0 + r_tile;                 // packed row within the episode
         const bool row_valid = r_local < rows_valid;
         // last visible key index; a padding row (beyond the episode's rows: its Q is zero fill or
         // another episode's) is never stored, so it takes everything unmasked rather than making its
         // warp mask every tile
-        const int bound = row_valid ? w.L + r_local / a.G : 0x3fffffff;
+        const int bound = row_valid ? w.L + (int)fast_div((uint32_t)r_local, a.div_g) : 0x3fffffff;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
-        const uint32_t t_o = t_lane + kColO + part * 32;
-        const uint32_t p_full0 = CTAS == 2 ? ptx::map_to_cta(bar_p_full, 0) : bar_p_full;
+        const uint32_t t_s = t_lane + (uint32_t)grp * 128;           // this group's score buffer
+        const uint32_t t_p = t_lane + kColP + (uint32_t)grp * 64;    // ... and its P buffer
+        const uint32_t t_o = t_lane + kColO + (uint32_t)grp * 64;
+        const uint32_t s_free0 = on_cta0(bar_s_free + 8 * grp);
+        const uint32_t p_full0 = on_cta0(bar_p_full + 8 * grp);
 
         float m_ref = -INFINITY;      // reference maximum (log2 domain) the exponentials use
         float l = 0.f;                // this thread's share of the running sum of exponentials
         bool ok = true;
         const uint64_t scale2 = ptx::pack2(a.scale_log2, a.scale_log2);
-        // Meeting of the kParts warps of this lane quarter (one phase of their barrier each): what any
-        // of them wrote to shared memory before its arrival is visible to the others after the wait.
+        // Meeting of the two warps of this lane quarter (one phase of their barrier each): what either
+        // wrote to shared memory before its arrival is visible to the other after the wait.
         auto meet = [&](uint32_t bar, int k) -> bool {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar + 8 * quarter);
             return warp_wait(bar + 8 * quarter, k & 1, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
         };
-        // A wait that gives way when a warp of this lane quarter has asked for a new reference:
+        // A wait that gives way when the other warp of this lane quarter has asked for a new reference:
         // 0 = the barrier completed, 1 = a request is pending, 2 = gave up (bounded wait expired).
+        // (Every lane probes once first: a barrier that is already complete costs one instruction.  The
+        // exponentials keep the sub-partition's queue to the SFU, the shared-memory and the barrier units
+        // full, so every dependent instruction on that path is worth ~100 cycles here.)
         auto wait_or_request = [&](uint32_t bar, uint32_t parity, int code) -> int {
+            if (__all_sync(0xffffffffu, ptx::mbar_try_wait(bar, parity))) return 0;
             int r = 0;
             if (lane == 0) {
                 if (s_req[quarter]) {
@@ -621,47 +635,27 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         // The exponentials of a row are taken against a reference m_ref that is fixed once (below) and
         // then left alone: the division by the row sum at the end makes any reference exact, and
         // floating point keeps the relative precision as long as nothing overflows, i.e. as long as
-        // no score exceeds the reference by more than 2^kRefHeadroom.  So the warps of a lane quarter
-        // do not talk to each other while they work and drift apart, which is what hides their
-        // barrier, TMEM and special-function latencies behind one another.  A thread that does meet
-        // such a score asks for a new reference: every warp of the quarter comes here at its next
-        // tile boundary (or out of a wait), with `released` = the first tile it has not handed to the
-        // tensor core yet (it has handed over all its tiles below) and `blocks` = how many 32-column
-        // blocks of that tile it has already written.  Nothing of a tile is consumed before all its
-        // parts are handed over and the products are issued in tile order, so the smallest `released`
-        // bounds what the accumulator holds; everybody then moves its own state to the new reference
-        // (a power-of-two factor, exact): running sum, its channels of O, and its blocks of the P
-        // tiles that are written but not yet consumed.
+        // no score exceeds the reference by more than 2^kRefHeadroom.  So the two threads of a row
+        // do not talk to each other while they work.  A thread that does meet such a score asks for a
+        // new reference: both warps of the quarter come here at their next tile boundary (or out of a
+        // wait), with `released` = the first tile it has not handed to the tensor core yet (it has
+        // handed over all its tiles below, and written nothing of that one).  Nothing of a tile is
+        // consumed before it is handed over and the products are issued in tile order, so the smaller
+        // `released` bounds what the accumulator holds; both then move their own state to the new
+        // reference (a power-of-two factor, exact): running sum, their channels of O, and their P
+        // tile if it is written but not yet consumed.
         int nrare = 0;                // meetings on bar_rare so far
         bool sum_published = false;   // this thread's share of the row sum is out for the final exchange
-        float* s_sum = s_xch + kParts * 128;
-        auto scale_p_block = [&](int t, int blk, float alpha) {
-            uint32_t pk[16];
-            const uint32_t t_pt = t_lane + (t % kScoreBufs) * 128 + half * 64 + blk * 32;
-            ptx::tmem_ld16(t_pt, pk);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                const float lo = __uint_as_float(pk[e] << 16) * alpha;
-                const float hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
-                pk[e] = ptx::pack_bf16x2(lo, hi);
-            }
-            ptx::tmem_st16(t_pt, pk);
-        };
-        auto move_reference = [&](int released, int blocks, bool mine, float want) -> bool {
-            s_cand[part * 128 + r_tile] = mine ? want : m_ref;
-            if (lane == 0) s_rel[quarter * kParts + part] = released;
+        auto move_reference = [&](int released, bool mine, float want) -> bool {
+            s_cand[grp * 128 + r_tile] = mine ? want : m_ref;
+            if (lane == 0) s_rel[quarter * kGroups + grp] = released;
             __syncwarp();
             if (lane == 0) s_req[quarter] = 1;
             if (!meet(bar_rare, nrare++)) return false;
-            int r_min = released;
-            float m_new = m_ref;
-#pragma unroll
-            for (int c = 0; c < kParts; ++c) {
-                r_min = min(r_min, s_rel[quarter * kParts + c]);
-                m_new = fmaxf(m_new, s_cand[c * 128 + r_tile]);
-            }
-            if (part == 0 && lane == 0) s_req[quarter] = 0;
+            const int r_min = min(s_rel[quarter * kGroups], s_rel[quarter * kGroups + 1]);
+            float m_new = fmaxf(s_cand[r_tile], s_cand[128 + r_tile]);
+            m_new = fmaxf(m_new, m_ref);
+            if (grp == 0 && lane == 0) s_req[quarter] = 0;
             // whole powers of two only, so that what is already rounded stays exact
             float alpha = 1.f;
             if (m_new > m_ref) {
@@ -683,113 +677,167 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                                    s_abort, lane))
                         return false;
                     ptx::fence_after_sync();
-                    uint32_t regs[32];              // this thread's 32 of the row's 128 channels
-                    ptx::tmem_ld32(t_o, regs);
-                    ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
-                    ptx::tmem_st32(t_o, regs);
+                    for (int hb = 0; hb < 2; ++hb) {            // this thread's 64 of the row's 128 channels
+                        uint32_t regs[32];
+                        ptx::tmem_ld32(t_o + hb * 32, regs);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
+                        ptx::tmem_st32(t_o + hb * 32, regs);
+                    }
                 }
-                // written, not consumed: this warp's tiles in [r_min, released) and the blocks of the
-                // tile it is working on
+                // written, not consumed: this warp's tiles in [r_min, released) (at most one: its P buffer)
                 for (int t = r_min; t < released; ++t) {
                     if ((t & 1) != grp) continue;
-                    scale_p_block(t, 0, alpha);
-                    scale_p_block(t, 1, alpha);
+#pragma unroll
+                    for (int blk = 0; blk < 4; ++blk) {
+                        uint32_t pk[16];
+                        ptx::tmem_ld16(t_p + blk * 16, pk);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float lo = __uint_as_float(pk[e] << 16) * alpha;
+                            const float hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
+                            pk[e] = ptx::pack_bf16x2(lo, hi);
+                        }
+                        ptx::tmem_st16(t_p + blk * 16, pk);
+                    }
                 }
-                for (int blk = 0; blk < blocks; ++blk) scale_p_block(released, blk, alpha);
                 l *= alpha;
                 ptx::tmem_st_wait();
                 ptx::fence_before_sync();
             }
             m_ref = m_new;
-            if (sum_published) s_sum[part * 128 + r_tile] = l;     // (ordered by the meeting below)
+            if (sum_published) s_sum[grp * 128 + r_tile] = l;     // (ordered by the meeting below)
             return meet(bar_rare, nrare++);
         };
 
         // The row's reference: the largest of its first 32 scores of the item's first tile (-inf: the
-        // row sees no key of this split, since the visible keys of a row are a prefix).  The thread that
-        // owns those columns reads it off and publishes it; nobody can ask for a new reference before.
-        if (part == 0) {
-            ok = warp_wait(bar_s_full, 0, kDevTimeoutSoftmaxS, a.status, s_abort, lane);
-            if (ok) {
-                ptx::fence_after_sync();
-                uint32_t s0[32];
-                ptx::tmem_ld32(t_lane, s0);
-                ptx::tmem_ld_wait();
-                const int lim = bound - w.j0 * kTileN;
-                if (lim < 31) mask32(s0, lim);
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-                rowmax32(s0, mx0, mx1, mx2, mx3);
-                m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
-                s_xch[r_tile] = m_ref;
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar_ref + 8 * quarter);
-            }
-        } else {
+        // row sees no key of this split, since the visible keys of a row are a prefix).  The group-0
+        // thread reads it off its first tile and publishes it; nobody can ask for a new reference
+        // before, so the group-1 thread simply waits for it.
+        if (grp == 1) {
             ok = warp_wait(bar_ref + 8 * quarter, 0, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
-            if (ok) m_ref = s_xch[r_tile];
+            if (ok) m_ref = s_ref[r_tile];
         }
 
         for (int jj = grp; jj < ntiles && ok; jj += 2) {
-            const int buf = jj % kScoreBufs;
+            const uint32_t use = (uint32_t)(jj >> 1);           // how often this group's buffers were used before
             while (ok) {
-                const int r = wait_or_request(bar_s_full + 8 * buf, (jj / kScoreBufs) & 1, kDevTimeoutSoftmaxS);
+                const int r = jj == 0 ? (warp_wait(bar_s_full, 0, kDevTimeoutSoftmaxS, a.status, s_abort, lane) ? 0 : 2)
+                                      : wait_or_request(bar_s_full + 8 * grp, use & 1, kDevTimeoutSoftmaxS);
                 if (r == 0) break;
-                ok = (r == 1) && move_reference(jj, 0, false, 0.f);
+                ok = (r == 1) && move_reference(jj, false, 0.f);
             }
             if (!ok) break;
             ptx::fence_after_sync();
-            if (half == 0 && quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(2 + jj);
+            if (quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(2 + jj);
 
+            // the row's 128 scores into registers; the score buffer goes back to the tensor core
+            uint32_t s[128];
 #pragma unroll
-            for (int blk = 0; blk < 2; ++blk) {
-                const int c0 = half * 64 + blk * 32;
-                const int lim = bound - (w.j0 + jj) * kTileN - c0;   // columns 0..lim of this block are visible
-                const bool no_mask = __all_sync(0xffffffffu, lim >= 31);
-                const uint32_t t_s = t_lane + buf * 128 + c0;        // P goes over this thread's own score columns only
+            for (int blk = 0; blk < 4; ++blk) ptx::tmem_ld32(t_s + blk * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[blk * 32]));
+            ptx::tmem_ld_wait();
+            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(56);
+            ptx::fence_before_sync();
+            if (ptx::elect_one()) {
+                if (CTAS == 2) ptx::mbar_arrive_cluster(s_free0); else ptx::mbar_arrive(s_free0);
+            }
 
-                uint32_t sA[32];
-                ptx::tmem_ld32(t_s, sA);
-                ptx::tmem_ld_wait();
-                if (!no_mask) mask32(sA, lim);  // -inf: masked keys (and stale slots) drop out
+            const int lim = bound - (w.j0 + jj) * kTileN;       // columns 0..lim of this tile are visible
+            if (!__all_sync(0xffffffffu, lim >= kTileN - 1)) {
+#pragma unroll
+                for (int blk = 0; blk < 4; ++blk) mask32(&s[blk * 32], lim - blk * 32);   // -inf: masked keys (and stale slots) drop out
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            rowmax32(&s[0], mx0, mx1, mx2, mx3);
+            if (jj == 0) {
+                m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
+                s_ref[r_tile] = m_ref;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_ref + 8 * quarter);
+            }
+#pragma unroll
+            for (int blk = 1; blk < 4; ++blk) rowmax32(&s[blk * 32], mx0, mx1, mx2, mx3);
+            const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
+            bool over = tmax > m_ref + kRefHeadroom;
+            while (ok && __any_sync(0xffffffffu, over)) {
+                ok = move_reference(jj, over, tmax);
+                over = tmax > m_ref + kRefHeadroom;
+            }
+            if (!ok) break;
+            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(57);
 
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-                rowmax32(sA, mx0, mx1, mx2, mx3);
-                const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
-                bool over = tmax > m_ref + kRefHeadroom;
-                while (ok && __any_sync(0xffffffffu, over)) {
-                    ok = move_reference(jj, blk, over, tmax);
-                    over = tmax > m_ref + kRefHeadroom;
+            // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P.  The P buffer is
+            // free once the product of tile jj - 2 has landed: this thread handed that tile over only a
+            // moment ago, so it asks after the first block of exponentials, not before.
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
+            uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
+            {
+                uint32_t pk[16];
+                exp32(&s[0], pk, scale2, negm2, sum2a, sum2b);
+                while (ok && jj >= 2) {
+                    const int r = wait_or_request(bar_pv_done + 8 * ((jj - 2) & 3), ((jj - 2) >> 2) & 1, kDevTimeoutSoftmaxO);
+                    if (r == 0) break;
+                    // (the meeting moves what is written and handed over; this block is still in
+                    // registers, so it follows by the same power of two)
+                    const float m_old = m_ref;
+                    ok = (r == 1) && move_reference(jj, false, 0.f);
+                    if (ok && m_ref != m_old) {
+                        const float alpha = (m_old == -INFINITY) ? 0.f : ptx::ex2(m_old - m_ref);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float lo = __uint_as_float(pk[e] << 16) * alpha;
+                            const float hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
+                            pk[e] = ptx::pack_bf16x2(lo, hi);
+                        }
+                        float a0, a1, b0, b1;
+                        ptx::unpack2(sum2a, a0, a1);
+                        ptx::unpack2(sum2b, b0, b1);
+                        sum2a = ptx::pack2(a0 * alpha, a1 * alpha);
+                        sum2b = ptx::pack2(b0 * alpha, b1 * alpha);
+                    }
                 }
                 if (!ok) break;
-
-                // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P over the S columns
-                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                const uint64_t negm2 = ptx::pack2(neg_m, neg_m);
-                uint64_t sum2a = ptx::pack2(0.f, 0.f), sum2b = sum2a;
-                exp32_store(sA, t_s, scale2, negm2, sum2a, sum2b);
+                ptx::fence_after_sync();
+                if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(58);
+                ptx::tmem_st16(t_p, pk);
+            }
+            {
+                // (the reference may have moved while waiting)
+                const float neg_m2 = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                const uint64_t negm2b = ptx::pack2(neg_m2, neg_m2);
+#pragma unroll
+                for (int blk = 1; blk < 4; ++blk) {
+                    uint32_t pk[16];
+                    exp32(&s[blk * 32], pk, scale2, negm2b, sum2a, sum2b);
+                    ptx::tmem_st16(t_p + blk * 16, pk);
+                }
+            }
+            {
                 float a0, a1, b0, b1;
                 ptx::unpack2(sum2a, a0, a1);
                 ptx::unpack2(sum2b, b0, b1);
                 l += (a0 + a1) + (b0 + b1);
             }
-            if (!ok) break;
+            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(59);
             ptx::tmem_st_wait();
             ptx::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-                if (CTAS == 2) ptx::mbar_arrive_cluster(p_full0 + 8 * buf); else ptx::mbar_arrive(p_full0 + 8 * buf);
+            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(63);
+            if (ptx::elect_one()) {
+                if (CTAS == 2) ptx::mbar_arrive_cluster(p_full0); else ptx::mbar_arrive(p_full0);
             }
-            if (half == 0 && quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(11 + jj);
+            if (quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(11 + jj);
         }
 
-        // All tiles handed over.  The row sum is the sum over the row's threads (same reference in
-        // all): they exchange it while the last product is still running.  A slower warp of the quarter
-        // may still ask for a new reference until it arrives here too; whoever serves such a request
-        // after publishing its share publishes the rescaled share again (inside move_reference).
+        // All tiles handed over.  The row sum is the sum of the row's two threads (same reference in
+        // both): they exchange it while the last product is still running.  The slower warp of the
+        // quarter may still ask for a new reference until it arrives here too; a warp that serves such
+        // a request after publishing its share publishes the rescaled share again (inside move_reference).
         if (ok) {
-            s_sum[part * 128 + r_tile] = l;
+            s_sum[grp * 128 + r_tile] = l;
             sum_published = true;
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
@@ -797,47 +845,50 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         while (ok) {
             const int r = wait_or_request(bar_xch + 8 * quarter, 0, kDevTimeoutSoftmaxX);
             if (r == 0) break;
-            ok = (r == 1) && move_reference(ntiles, 0, false, 0.f);
+            ok = (r == 1) && move_reference(ntiles, false, 0.f);
         }
         // nobody of the quarter can ask any more; the last product
         if (ok) ok = warp_wait(bar_o_full, 0, kDevTimeoutSoftmaxO, a.status, s_abort, lane);
         if (ok) {
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(60);
-            l = 0.f;
-#pragma unroll
-            for (int c = 0; c < kParts; ++c) l += s_sum[c * 128 + r_tile];
+            l = s_sum[r_tile] + s_sum[128 + r_tile];
             // Epilogue: O/l goes out through shared memory so that global stores are whole
             // 128-byte lines.  The K ring is dead (its last consumer has completed); each warp
-            // stages its 32 rows x 32 channels there, rows 144 bytes apart.
+            // stages 32 rows x 32 channels there at a time, rows 144 bytes apart.
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             const int wrow0 = quarter << 5;
             uint8_t* stage = smem_gen + kSmemKOff + (warp - 4) * (32 * 144);
             const int first_row = row0 + wrow0;                              // episode-local
             const int rows_here = rows_valid - first_row;                    // may be <= 0 or > 32
             const long prow0 = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + first_row;
-            float* gbase = a.o_part + prow0 * 128 + part * 32;
-            uint32_t regs[32];
-            ptx::tmem_ld32(t_o, regs);
-            ptx::tmem_ld_wait();
-            float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
 #pragma unroll
-            for (int e = 0; e < 32; e += 4)
-                srow[e >> 2] = make_float4(__uint_as_float(regs[e]) * inv, __uint_as_float(regs[e + 1]) * inv,
-                                           __uint_as_float(regs[e + 2]) * inv, __uint_as_float(regs[e + 3]) * inv);
-            __syncwarp();
+            for (int hb = 0; hb < 2; ++hb) {
+                float* gbase = a.o_part + prow0 * 128 + grp * 64 + hb * 32;
+                uint32_t regs[32];
+                ptx::tmem_ld32(t_o + hb * 32, regs);
+                ptx::tmem_ld_wait();
+                float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int r = i * 4 + (lane >> 3);
-                if (r < rows_here) {
-                    const float4 v = *reinterpret_cast<const float4*>(stage + r * 144 + (lane & 7) * 16);
-                    *reinterpret_cast<float4*>(gbase + (long)r * 128 + (lane & 7) * 4) = v;
+                for (int e = 0; e < 32; e += 4)
+                    srow[e >> 2] = make_float4(__uint_as_float(regs[e]) * inv, __uint_as_float(regs[e + 1]) * inv,
+                                               __uint_as_float(regs[e + 2]) * inv, __uint_as_float(regs[e + 3]) * inv);
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = i * 4 + (lane >> 3);
+                    if (r < rows_here) {
+                        const float4 v = *reinterpret_cast<const float4*>(stage + r * 144 + (lane & 7) * 16);
+                        *reinterpret_cast<float4*>(gbase + (long)r * 128 + (lane & 7) * 4) = v;
+                    }
                 }
+                __syncwarp();
             }
-            if (row_valid && part == 0)
+            if (row_valid && grp == 0)
                 a.lse_part[prow0 + lane] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
             if (warp == 4 && lane == 0) EVLN_STAMP(61);
         }
+    }
     }
 
     // ---- teardown: nobody leaves while the other CTA may still touch this CTA's memory ----
