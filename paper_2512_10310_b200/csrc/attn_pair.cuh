@@ -12,7 +12,7 @@
 // query rows.  The item's normalised partial outputs + log-sum-exps go to the workspace that
 // the combine kernel merges.
 //
-// Per CTA (384 threads, 1 CTA/SM, ~199 KB shared memory, all 512 TMEM columns):
+// Per CTA (640 threads, 1 CTA/SM, ~199 KB shared memory, all 512 TMEM columns):
 //   warp 0      TMA producer: the CTA's Q tile once, then its K / V half tiles through two
 //               5-deep rings of 16 KB stages (128B-swizzled); no multicast anywhere.  Bytes are
 //               counted on barriers of CTA 0, where the MMA threads wait.
@@ -21,19 +21,21 @@
 //   warp 2      (CTA 0) product issuer: O += P_j V_j (A = P_j from tensor memory, buffer j % 2)
 //               as soon as P_j is written.  Scores and products have buffers of their own, so
 //               neither instruction stream waits for the other.
-//   warps 4-11  softmax + epilogue, two warps per TMEM lane quarter (= per SM sub-partition), one
-//               thread per query row.  The warps of group 0 take the even KV tiles of the item,
-//               those of group 1 the odd ones: a thread pulls the 128 scores of its row into
-//               registers, gives the score buffer back at once, and then works through its 128
-//               exponentials while the other warp of the sub-partition is in another phase of
-//               another tile (a tile's exponentials keep the 4 SFU lanes of a sub-partition busy
-//               for as long as its MMAs keep the tensor pipe busy, so that unit must not idle).
-//               The exponentials of a row are taken against a reference that the group-0 thread
-//               reads off the first 32 scores of the first tile and passes to the other thread
-//               through shared memory; the two talk to each other again only if a later score
-//               exceeds it by more than 2^64 (then O, the row sums and the pending P tiles are
-//               rescaled by a power of two); the final division by the row sum makes any
-//               reference exact.
+//   warps 4-19  softmax + epilogue, four warps per TMEM lane quarter (= per SM sub-partition), two
+//               threads per query row and tile.  The warps of group 0 take the even KV tiles of the
+//               item, those of group 1 the odd ones; within a group a thread owns 64 of the 128
+//               score columns of its row: it pulls them into registers, gives the score buffer back
+//               at once, and then works through its 64 exponentials while the other three warps
+//               of the sub-partition are in other phases of their tiles.  (One warp needs ~2.5 K
+//               cycles of mostly latency for its share of a tile, the tensor pipe ~1 K for the
+//               tile's MMAs: four warps in flight per sub-partition are what hides the chain; a
+//               tile's exponentials also keep the 4 SFU lanes of a sub-partition busy for ~1 K
+//               cycles, so that unit must not idle either.)  The exponentials of a row are taken
+//               against a reference that one thread of the row reads off the first 32 scores of
+//               the first tile and passes to the other three through shared memory; they talk to
+//               each other again only if a later score exceeds it by more than 2^64 (then O, the
+//               row sums and the pending P tiles are rescaled by a power of two); the final
+//               division by the row sum makes any reference exact.
 //   warp 3      sets up barriers (with warp 2), then idles.
 // TMEM columns: scores S_b at 128 b, b = 0..1; P_b (128 keys as 64 columns of packed bf16 pairs) at
 // 256 + 64 b; O at 384.
@@ -51,12 +53,12 @@
 
 namespace evln {
 
-constexpr int kTcThreads = 384;
-constexpr int kGroups = 2;                            // softmax threads per query row: one per tile parity
+constexpr int kTcThreads = 640;
+constexpr int kParts = 4;                             // softmax threads per query row: tile parity x column half
 constexpr int kTileBytes = kTileM * 128 * 2;          // Q tile: 128 rows x 128 channels x bf16
 constexpr int kHalfBytes = kTileBytes / 2;            // 16 KB: a 64-channel half of Q; a K or V half tile
 constexpr int kSmemBarBytes = 384;
-constexpr int kSmemXchBytes = 128 * 4 + 2 * kGroups * 128 * 4 + 128;
+constexpr int kSmemXchBytes = 128 * 4 + 2 * kParts * 128 * 4 + 128;
 
 // Shared-memory plan of a CTA.  CTAS = 2: the CTA of a pair stages half tiles (16 KB) through two
 // 5-deep rings.  CTAS = 1: a CTA on its own stages whole K / V tiles (32 KB: two 64-channel blocks
@@ -71,18 +73,24 @@ struct SmemPlan {
     static constexpr int kVOff = kKOff + kKStages * kStageBytes;
     static constexpr int kBarOff = kVOff + kVStages * kStageBytes;
     static constexpr int kRefOff = kBarOff + kSmemBarBytes;          // float [128 rows]: published references
-    static constexpr int kSumOff = kRefOff + 128 * 4;                // float [kGroups][128 rows]: row-sum shares
-    static constexpr int kCandOff = kSumOff + kGroups * 128 * 4;     // float [kGroups][128 rows]: reference requests
-    static constexpr int kReqOff = kCandOff + kGroups * 128 * 4;     // int [4] request flags, int [4][kGroups] released tiles
+    static constexpr int kSumOff = kRefOff + 128 * 4;                // float [kParts][128 rows]: row-sum shares
+    static constexpr int kCandOff = kSumOff + kParts * 128 * 4;      // float [kParts][128 rows]: reference requests
+    static constexpr int kReqOff = kCandOff + kParts * 128 * 4;      // int [4] request flags, int [4][kParts] released tiles
     static constexpr int kBytes = kRefOff + kSmemXchBytes + 1024;    // + slack to align to 1024
-    static_assert(kKStages * kStageBytes >= 8 * 32 * 144, "the epilogue stages its rows in the K ring");
+    static_assert(kKStages * kStageBytes >= 16 * 32 * 144, "the epilogue stages its rows in the K ring");
     static_assert(kBytes <= 227 * 1024, "shared memory per CTA");
 };
 constexpr int kTcSmemBytes = SmemPlan<2>::kBytes;
 constexpr int kSoloSmemBytes = SmemPlan<1>::kBytes;
 constexpr long long kWaitLimitCycles = 2000000000LL;  // ~1 s at boost clocks
 constexpr int kScoreBufs = 2;
-constexpr int kRegsIssue = 80, kRegsSoftmax = 208;    // per thread, after the set-up (4 + 8 warps: 62 K of 64 K registers)
+// Registers per thread after the set-up.  setmaxnreg moves registers inside the pool the CTA got at
+// launch (kTcThreads x the kernel's register count, kRegsLaunch): what the issue warpgroup gives up
+// must cover what the softmax warpgroups take, or their request waits for ever.  The host checks
+// the compiled register count against kRegsLaunch before the first launch.
+constexpr int kRegsLaunch = 96, kRegsIssue = 32, kRegsSoftmax = 112;
+static_assert((kRegsLaunch - kRegsIssue) * 128 >= (kRegsSoftmax - kRegsLaunch) * (kTcThreads - 128), "register pool of a CTA");
+static_assert(kRegsLaunch * kTcThreads <= 65536, "register file of an SM");
 constexpr uint32_t kColP = 256;
 constexpr uint32_t kColO = 384;
 #ifndef EVLN_REF_HEADROOM
@@ -294,13 +302,13 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     const uint32_t bar_pv_done = bar_s_full + 8 * kScoreBufs;    // [4] PV of tile j landed: barrier j % 4
     const uint32_t bar_o_full = bar_pv_done + 32;                // last PV landed
     const uint32_t bar_ref = bar_o_full + 8;                     // [4] the rows' references are published
-    const uint32_t bar_xch = bar_ref + 32;                       // [4] the two warps of a lane quarter meet here (row sums)
+    const uint32_t bar_xch = bar_ref + 32;                       // [4] the four warps of a lane quarter meet here (row sums)
     const uint32_t bar_rare = bar_xch + 32;                      // [4] ... and here when a row's reference has to move
     const uint32_t tmem_slot = bar_rare + 32;                    // uint32
     constexpr int kBarsCtas = 1 + kKStages + kVStages;                                 // arrival count CTAS
     constexpr int kBarsSoft = 2 * kScoreBufs;                                          // one per softmax warp of the tile
     constexpr int kBarsOne = kKStages + kVStages + kScoreBufs + 4 + 1 + 4;             // count 1
-    constexpr int kNumBars = kBarsCtas + kBarsSoft + kBarsOne + 8;                     // + xch, rare: kGroups
+    constexpr int kNumBars = kBarsCtas + kBarsSoft + kBarsOne + 8;                     // + xch, rare: kParts
     static_assert(8 * kNumBars + 8 <= kSmemBarBytes, "barrier area");
     static_assert(kNumBars <= 64, "one thread of warps 2-3 per barrier");
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem_gen + (tmem_slot - smem_base));
@@ -309,7 +317,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     float* s_sum = reinterpret_cast<float*>(smem_gen + Plan::kSumOff);
     float* s_cand = reinterpret_cast<float*>(smem_gen + Plan::kCandOff);
     volatile int* s_req = reinterpret_cast<volatile int*>(smem_gen + Plan::kReqOff);        // [4]
-    volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + Plan::kReqOff) + 4;    // [4][kGroups]
+    volatile int* s_rel = reinterpret_cast<volatile int*>(smem_gen + Plan::kReqOff) + 4;    // [4][kParts]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;   // 0: issues the MMAs, owns the "(CTA 0)" barriers
@@ -368,9 +376,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         if (i < kNumBars) {
             int count = 1;
             if (i < kBarsCtas) count = CTAS;                                   // q_full, k_full, v_full
-            else if (i < kBarsCtas + kBarsSoft) count = CTAS * quarters;       // s_free, p_full: the tile's softmax warps
+            else if (i < kBarsCtas + kBarsSoft) count = CTAS * quarters * 2;   // s_free, p_full: the tile's softmax warps
             else if (i < kBarsCtas + kBarsSoft + kBarsOne) count = 1;          // k_empty .. ref
-            else count = kGroups;                                              // xch, rare
+            else count = kParts;                                               // xch, rare
             ptx::mbar_init(bar_base + 8 * i, count);
             ptx::fence_barrier_init();
         }
@@ -575,7 +583,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     if ((warp & 3) < quarters) {
         // ================= softmax + epilogue =================
         const int quarter = warp & 3;                      // TMEM lane quarter of this warp
-        const int grp = (warp - 4) >> 2;                   // its KV tiles: grp, grp + 2, ...; its 64 channels of O
+        const int part = (warp - 4) >> 2;                  // its 32 channels of O (epilogue, rescales)
+        const int grp = part >> 1;                         // its KV tiles: grp, grp + 2, ...
+        const int half = part & 1;                         // its score columns: [64 half, +64), two blocks of 32
         const int r_tile = (quarter << 5) + lane;          // row within the tile = TMEM lane
         const int r_local = row0 + r_tile;                 // packed row within the episode
         const bool row_valid = r_local < rows_valid;
@@ -584,9 +594,9 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         // warp mask every tile
         const int bound = row_valid ? w.L + (int)fast_div((uint32_t)r_local, a.div_g) : 0x3fffffff;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
-        const uint32_t t_s = t_lane + (uint32_t)grp * 128;           // this group's score buffer
-        const uint32_t t_p = t_lane + kColP + (uint32_t)grp * 64;    // ... and its P buffer
-        const uint32_t t_o = t_lane + kColO + (uint32_t)grp * 64;
+        const uint32_t t_s = t_lane + (uint32_t)grp * 128 + (uint32_t)half * 64;          // its half of the group's score buffer
+        const uint32_t t_p = t_lane + kColP + (uint32_t)grp * 64 + (uint32_t)half * 32;   // ... and of its P buffer
+        const uint32_t t_o = t_lane + kColO + (uint32_t)part * 32;
         const uint32_t s_free0 = on_cta0(bar_s_free + 8 * grp);
         const uint32_t p_full0 = on_cta0(bar_p_full + 8 * grp);
 
@@ -594,14 +604,14 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         float l = 0.f;                // this thread's share of the running sum of exponentials
         bool ok = true;
         const uint64_t scale2 = ptx::pack2(a.scale_log2, a.scale_log2);
-        // Meeting of the two warps of this lane quarter (one phase of their barrier each): what either
-        // wrote to shared memory before its arrival is visible to the other after the wait.
+        // Meeting of the four warps of this lane quarter (one phase of their barrier each): what any of
+        // them wrote to shared memory before its arrival is visible to the others after the wait.
         auto meet = [&](uint32_t bar, int k) -> bool {
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar + 8 * quarter);
             return warp_wait(bar + 8 * quarter, k & 1, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
         };
-        // A wait that gives way when the other warp of this lane quarter has asked for a new reference:
+        // A wait that gives way when a warp of this lane quarter has asked for a new reference:
         // 0 = the barrier completed, 1 = a request is pending, 2 = gave up (bounded wait expired).
         // (Every lane probes once first: a barrier that is already complete costs one instruction.  The
         // exponentials keep the sub-partition's queue to the SFU, the shared-memory and the barrier units
@@ -635,27 +645,31 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         // The exponentials of a row are taken against a reference m_ref that is fixed once (below) and
         // then left alone: the division by the row sum at the end makes any reference exact, and
         // floating point keeps the relative precision as long as nothing overflows, i.e. as long as
-        // no score exceeds the reference by more than 2^kRefHeadroom.  So the two threads of a row
+        // no score exceeds the reference by more than 2^kRefHeadroom.  So the four threads of a row
         // do not talk to each other while they work.  A thread that does meet such a score asks for a
-        // new reference: both warps of the quarter come here at their next tile boundary (or out of a
+        // new reference: all warps of the quarter come here at their next tile boundary (or out of a
         // wait), with `released` = the first tile it has not handed to the tensor core yet (it has
         // handed over all its tiles below, and written nothing of that one).  Nothing of a tile is
-        // consumed before it is handed over and the products are issued in tile order, so the smaller
-        // `released` bounds what the accumulator holds; both then move their own state to the new
+        // consumed before it is handed over and the products are issued in tile order, so the smallest
+        // `released` bounds what the accumulator holds; all then move their own state to the new
         // reference (a power-of-two factor, exact): running sum, their channels of O, and their P
         // tile if it is written but not yet consumed.
         int nrare = 0;                // meetings on bar_rare so far
         bool sum_published = false;   // this thread's share of the row sum is out for the final exchange
         auto move_reference = [&](int released, bool mine, float want) -> bool {
-            s_cand[grp * 128 + r_tile] = mine ? want : m_ref;
-            if (lane == 0) s_rel[quarter * kGroups + grp] = released;
+            s_cand[part * 128 + r_tile] = mine ? want : m_ref;
+            if (lane == 0) s_rel[quarter * kParts + part] = released;
             __syncwarp();
             if (lane == 0) s_req[quarter] = 1;
             if (!meet(bar_rare, nrare++)) return false;
-            const int r_min = min(s_rel[quarter * kGroups], s_rel[quarter * kGroups + 1]);
-            float m_new = fmaxf(s_cand[r_tile], s_cand[128 + r_tile]);
-            m_new = fmaxf(m_new, m_ref);
-            if (grp == 0 && lane == 0) s_req[quarter] = 0;
+            int r_min = released;
+            float m_new = m_ref;
+#pragma unroll
+            for (int c = 0; c < kParts; ++c) {
+                r_min = min(r_min, s_rel[quarter * kParts + c]);
+                m_new = fmaxf(m_new, s_cand[c * 128 + r_tile]);
+            }
+            if (part == 0 && lane == 0) s_req[quarter] = 0;
             // whole powers of two only, so that what is already rounded stays exact
             float alpha = 1.f;
             if (m_new > m_ref) {
@@ -677,21 +691,18 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                                    s_abort, lane))
                         return false;
                     ptx::fence_after_sync();
+                    uint32_t regs[32];              // this thread's 32 of the row's 128 channels
+                    ptx::tmem_ld32(t_o, regs);
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int hb = 0; hb < 2; ++hb) {            // this thread's 64 of the row's 128 channels
-                        uint32_t regs[32];
-                        ptx::tmem_ld32(t_o + hb * 32, regs);
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
-                        ptx::tmem_st32(t_o + hb * 32, regs);
-                    }
+                    for (int e = 0; e < 32; ++e) regs[e] = __float_as_uint(__uint_as_float(regs[e]) * alpha);
+                    ptx::tmem_st32(t_o, regs);
                 }
-                // written, not consumed: this warp's tiles in [r_min, released) (at most one: its P buffer)
+                // written, not consumed: this warp's tiles in [r_min, released) (at most one: its half of the P buffer)
                 for (int t = r_min; t < released; ++t) {
                     if ((t & 1) != grp) continue;
 #pragma unroll
-                    for (int blk = 0; blk < 4; ++blk) {
+                    for (int blk = 0; blk < 2; ++blk) {
                         uint32_t pk[16];
                         ptx::tmem_ld16(t_p + blk * 16, pk);
                         ptx::tmem_ld_wait();
@@ -709,15 +720,15 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 ptx::fence_before_sync();
             }
             m_ref = m_new;
-            if (sum_published) s_sum[grp * 128 + r_tile] = l;     // (ordered by the meeting below)
+            if (sum_published) s_sum[part * 128 + r_tile] = l;    // (ordered by the meeting below)
             return meet(bar_rare, nrare++);
         };
 
         // The row's reference: the largest of its first 32 scores of the item's first tile (-inf: the
-        // row sees no key of this split, since the visible keys of a row are a prefix).  The group-0
-        // thread reads it off its first tile and publishes it; nobody can ask for a new reference
-        // before, so the group-1 thread simply waits for it.
-        if (grp == 1) {
+        // row sees no key of this split, since the visible keys of a row are a prefix).  The
+        // thread that owns those columns reads it off and publishes it; nobody can ask for a new
+        // reference before, so the other threads of the row simply wait for it.
+        if (part != 0) {
             ok = warp_wait(bar_ref + 8 * quarter, 0, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
             if (ok) m_ref = s_ref[r_tile];
         }
@@ -725,41 +736,41 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         for (int jj = grp; jj < ntiles && ok; jj += 2) {
             const uint32_t use = (uint32_t)(jj >> 1);           // how often this group's buffers were used before
             while (ok) {
-                const int r = jj == 0 ? (warp_wait(bar_s_full, 0, kDevTimeoutSoftmaxS, a.status, s_abort, lane) ? 0 : 2)
-                                      : wait_or_request(bar_s_full + 8 * grp, use & 1, kDevTimeoutSoftmaxS);
+                const int r = (jj == 0 && part == 0)
+                                  ? (warp_wait(bar_s_full, 0, kDevTimeoutSoftmaxS, a.status, s_abort, lane) ? 0 : 2)
+                                  : wait_or_request(bar_s_full + 8 * grp, use & 1, kDevTimeoutSoftmaxS);
                 if (r == 0) break;
                 ok = (r == 1) && move_reference(jj, false, 0.f);
             }
             if (!ok) break;
             ptx::fence_after_sync();
-            if (quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(2 + jj);
+            if (quarter == 0 && half == 0 && lane == 0 && jj < 9) EVLN_STAMP(2 + jj);
 
-            // the row's 128 scores into registers; the score buffer goes back to the tensor core
-            uint32_t s[128];
+            // this thread's 64 scores of the row into registers; the score buffer goes back to the tensor core
+            uint32_t s[64];
 #pragma unroll
-            for (int blk = 0; blk < 4; ++blk) ptx::tmem_ld32(t_s + blk * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[blk * 32]));
+            for (int blk = 0; blk < 2; ++blk) ptx::tmem_ld32(t_s + blk * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[blk * 32]));
             ptx::tmem_ld_wait();
-            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(56);
+            if (quarter == 0 && half == 0 && lane == 0 && jj == 4) EVLN_STAMP(56);
             ptx::fence_before_sync();
             if (ptx::elect_one()) {
                 if (CTAS == 2) ptx::mbar_arrive_cluster(s_free0); else ptx::mbar_arrive(s_free0);
             }
 
-            const int lim = bound - (w.j0 + jj) * kTileN;       // columns 0..lim of this tile are visible
-            if (!__all_sync(0xffffffffu, lim >= kTileN - 1)) {
+            const int lim = bound - (w.j0 + jj) * kTileN - half * 64;   // columns 0..lim of this thread's 64 are visible
+            if (!__all_sync(0xffffffffu, lim >= 63)) {
 #pragma unroll
-                for (int blk = 0; blk < 4; ++blk) mask32(&s[blk * 32], lim - blk * 32);   // -inf: masked keys (and stale slots) drop out
+                for (int blk = 0; blk < 2; ++blk) mask32(&s[blk * 32], lim - blk * 32);   // -inf: masked keys (and stale slots) drop out
             }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
             rowmax32(&s[0], mx0, mx1, mx2, mx3);
-            if (jj == 0) {
+            if (jj == 0 && part == 0) {
                 m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;   // scale > 0
                 s_ref[r_tile] = m_ref;
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(bar_ref + 8 * quarter);
             }
-#pragma unroll
-            for (int blk = 1; blk < 4; ++blk) rowmax32(&s[blk * 32], mx0, mx1, mx2, mx3);
+            rowmax32(&s[32], mx0, mx1, mx2, mx3);
             const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
             bool over = tmax > m_ref + kRefHeadroom;
             while (ok && __any_sync(0xffffffffu, over)) {
@@ -767,7 +778,7 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 over = tmax > m_ref + kRefHeadroom;
             }
             if (!ok) break;
-            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(57);
+            if (quarter == 0 && half == 0 && lane == 0 && jj == 4) EVLN_STAMP(57);
 
             // P = 2^(s*scale_log2 - m_ref) (packed FMA), row sum (packed add), bf16 P.  The P buffer is
             // free once the product of tile jj - 2 has landed: this thread handed that tile over only a
@@ -802,19 +813,16 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 }
                 if (!ok) break;
                 ptx::fence_after_sync();
-                if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(58);
+                if (quarter == 0 && half == 0 && lane == 0 && jj == 4) EVLN_STAMP(58);
                 ptx::tmem_st16(t_p, pk);
             }
             {
                 // (the reference may have moved while waiting)
                 const float neg_m2 = (m_ref == -INFINITY) ? 0.f : -m_ref;
                 const uint64_t negm2b = ptx::pack2(neg_m2, neg_m2);
-#pragma unroll
-                for (int blk = 1; blk < 4; ++blk) {
-                    uint32_t pk[16];
-                    exp32(&s[blk * 32], pk, scale2, negm2b, sum2a, sum2b);
-                    ptx::tmem_st16(t_p + blk * 16, pk);
-                }
+                uint32_t pk[16];
+                exp32(&s[32], pk, scale2, negm2b, sum2a, sum2b);
+                ptx::tmem_st16(t_p + 16, pk);
             }
             {
                 float a0, a1, b0, b1;
@@ -822,22 +830,22 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 ptx::unpack2(sum2b, b0, b1);
                 l += (a0 + a1) + (b0 + b1);
             }
-            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(59);
+            if (quarter == 0 && half == 0 && lane == 0 && jj == 4) EVLN_STAMP(59);
             ptx::tmem_st_wait();
             ptx::fence_before_sync();
-            if (quarter == 0 && lane == 0 && jj == 4) EVLN_STAMP(63);
+            if (quarter == 0 && half == 0 && lane == 0 && jj == 4) EVLN_STAMP(63);
             if (ptx::elect_one()) {
                 if (CTAS == 2) ptx::mbar_arrive_cluster(p_full0); else ptx::mbar_arrive(p_full0);
             }
-            if (quarter == 0 && lane == 0 && jj < 9) EVLN_STAMP(11 + jj);
+            if (quarter == 0 && half == 0 && lane == 0 && jj < 9) EVLN_STAMP(11 + jj);
         }
 
-        // All tiles handed over.  The row sum is the sum of the row's two threads (same reference in
-        // both): they exchange it while the last product is still running.  The slower warp of the
+        // All tiles handed over.  The row sum is the sum of the row's four threads (same reference in
+        // all): they exchange it while the last product is still running.  A slower warp of the
         // quarter may still ask for a new reference until it arrives here too; a warp that serves such
         // a request after publishing its share publishes the rescaled share again (inside move_reference).
         if (ok) {
-            s_sum[grp * 128 + r_tile] = l;
+            s_sum[part * 128 + r_tile] = l;
             sum_published = true;
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar_xch + 8 * quarter);
@@ -852,21 +860,20 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         if (ok) {
             ptx::fence_after_sync();
             if (warp == 4 && lane == 0) EVLN_STAMP(60);
-            l = s_sum[r_tile] + s_sum[128 + r_tile];
+            l = (s_sum[r_tile] + s_sum[128 + r_tile]) + (s_sum[256 + r_tile] + s_sum[384 + r_tile]);
             // Epilogue: O/l goes out through shared memory so that global stores are whole
             // 128-byte lines.  The K ring is dead (its last consumer has completed); each warp
-            // stages 32 rows x 32 channels there at a time, rows 144 bytes apart.
+            // stages its 32 rows x 32 channels there, rows 144 bytes apart.
             const float inv = (l > 0.f) ? 1.f / l : 0.f;
             const int wrow0 = quarter << 5;
             uint8_t* stage = smem_gen + kSmemKOff + (warp - 4) * (32 * 144);
             const int first_row = row0 + wrow0;                              // episode-local
             const int rows_here = rows_valid - first_row;                    // may be <= 0 or > 32
             const long prow0 = ((long)w.slot * a.Hkv + w.g) * a.rows + w.row_base + first_row;
-#pragma unroll
-            for (int hb = 0; hb < 2; ++hb) {
-                float* gbase = a.o_part + prow0 * 128 + grp * 64 + hb * 32;
+            {
+                float* gbase = a.o_part + prow0 * 128 + part * 32;
                 uint32_t regs[32];
-                ptx::tmem_ld32(t_o + hb * 32, regs);
+                ptx::tmem_ld32(t_o, regs);
                 ptx::tmem_ld_wait();
                 float4* srow = reinterpret_cast<float4*>(stage + lane * 144);
 #pragma unroll
@@ -882,9 +889,8 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                         *reinterpret_cast<float4*>(gbase + (long)r * 128 + (lane & 7) * 4) = v;
                     }
                 }
-                __syncwarp();
             }
-            if (row_valid && grp == 0)
+            if (row_valid && part == 0)
                 a.lse_part[prow0 + lane] = (l > 0.f) ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
             if (warp == 4 && lane == 0) EVLN_STAMP(61);
         }

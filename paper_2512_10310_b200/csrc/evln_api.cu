@@ -85,6 +85,21 @@ cudaError_t launch_pair_pdl(void (*kernel)(KArgs...), dim3 grid, size_t smem, cu
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// The attention kernels move registers between their warpgroups (setmaxnreg) inside the pool a CTA
+// gets at launch; a request the pool cannot serve would wait for ever.  The plan in attn_pair.cuh is
+// made for kRegsLaunch registers per thread: refuse to run a build that came out differently.
+bool attention_register_pool_ok()
+{
+    cudaFuncAttributes fa;
+    const void* kernels[3] = {(const void*)attn_pair_kernel<false, NoLens>, (const void*)attn_pair_kernel<true, BatchLens>,
+                              (const void*)attn_solo_kernel};
+    for (const void* k : kernels) {
+        if (cudaFuncGetAttributes(&fa, k) != cudaSuccess) return false;
+        if (fa.numRegs != kRegsLaunch) return false;
+    }
+    return true;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int elem_bytes(int dtype) { return dtype == EVLN_BF16 ? 2 : 4; }
@@ -343,6 +358,11 @@ evlnStatus_t evlnCreate(evlnHandle_t* handle, int device)
                                  kTcSmemBytes);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(attn_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSoloSmemBytes);
+    if (e == cudaSuccess && !attention_register_pool_ok()) {
+        cudaFree(h->d_status);
+        delete h;
+        return EVLN_NOT_SUPPORTED;
+    }
     if (e != cudaSuccess) {
         if (h->d_status) cudaFree(h->d_status);
         delete h;
@@ -867,6 +887,7 @@ evlnStatus_t noalloc_setup(int device, NoAllocDevice** out)
         if (e != cudaSuccess) return EVLN_CUDA_ERROR;
         e = cudaFuncSetAttribute(attn_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSoloSmemBytes);
         if (e != cudaSuccess) return EVLN_CUDA_ERROR;
+        if (!attention_register_pool_ok()) return EVLN_NOT_SUPPORTED;
         d->ctx.device = device;
         d->ctx.num_sms = prop.multiProcessorCount;
         d->ctx.last_cuda_error = 0;
