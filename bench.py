@@ -47,13 +47,14 @@ def load_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML while timed regions run (`recording` set)."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.004):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop_evt = threading.Event()
+        self.recording = threading.Event()
         self.ok = False
         try:
             import pynvml
@@ -76,6 +77,9 @@ class ClockSampler(threading.Thread):
             getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
         }
         while not self._stop_evt.is_set():
+            if not self.recording.is_set():
+                time.sleep(self.period)
+                continue
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
                 try:
@@ -111,48 +115,52 @@ def physical_gpu_index(local_index: int) -> int:
 # our arm
 # ------------------------------------------------------------------------------------------------
 
-# DRAM bytes (read + write) of one attention launch at this workload, from the ncu capture that
-# profiles/attn_pair_kernel_step_7b_L4096.md summarises.  The counters belong to the kernel sources
-# as they were then: once one of them changes, the figure is withheld until it is taken again.
-K2_DRAM_BYTES_PER_LAUNCH = 10_252_800
+MIN_REPLAYS = 200           # every timed graph is replayed at least this often, whatever --steps says
 K2_SOURCES = ("attn_pair.cuh", "ptx_sm100.cuh", "common.cuh")
-K2_SOURCES_SHA256 = "6f7c38c01567322f232d5812107eed20469ee785406c52cd6ea74afc6b542220"
+K2_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "attn_pair_kernel_step_7b_L4096.traffic.txt")
 
 
 def attention_dram_traffic():
+    """DRAM bytes (read + write) of one attention launch at the headline workload, as counted by the
+    last ncu capture.  The figure belongs to the kernel sources as they were then (their SHA-256 is
+    stored beside it): once one of them changes it is withheld until the counters are taken again."""
     import hashlib
     h = hashlib.sha256()
-    src = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2512_10310_b200", "csrc")
+    src = os.path.join(ROOT, "paper_2512_10310_b200", "csrc")
     try:
         for name in K2_SOURCES:
             with open(os.path.join(src, name), "rb") as fh:
                 h.update(fh.read())
-    except OSError:
+        rec = dict(line.strip().split("=", 1) for line in open(K2_TRAFFIC_FILE) if "=" in line and not line.startswith("#"))
+        return int(rec["dram_bytes_per_launch"]) if rec.get("sha256") == h.hexdigest() else None
+    except (OSError, KeyError, ValueError):
         return None
-    return K2_DRAM_BYTES_PER_LAUNCH if h.hexdigest() == K2_SOURCES_SHA256 else None
 
 
 class LayerRing:
-    """Device buffers of RING_LAYERS independent layers of the workload + pinned host copies."""
+    """Device buffers of independent layers of one workload (+ pinned host copies when asked for).
+    One position table serves all layers, as in a model: it is made once per pass over the ring."""
 
-    def __init__(self, B, handle, cfg, dev, layers, random_device_inputs=False):
+    def __init__(self, B, handle, cfg, dev, layers, host_copies=False):
         self.B, self.h, self.cfg, self.dev = B, handle, cfg, dev
         L, n, Hq, Hkv, D = cfg.cache_len, cfg.num_new, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
-        self.p = B.step_params(cfg.dtype, Hq, Hkv, D, L, n, L + n, cfg.rope_theta)
+        self.table = torch.empty(max(B.evlnRopeTableBytes(D, n), 16), dtype=torch.uint8, device=dev)
+        self.p = B.step_params(cfg.dtype, Hq, Hkv, D, L, n, L + n, cfg.rope_theta, rope_table=self.table,
+                               rope_table_first_pos=L, rope_table_count=n)
         qbytes = B.evlnStepQRotSize(handle, self.p)
         wbytes = B.evlnStepWorkspaceSize(handle, self.p)
         self.splits = B.evlnStepNumSplits(handle, self.p)
         self.layers = []
         dt = cfg.torch_dtype
         for l in range(layers):
-            if random_device_inputs:
-                # same distribution, drawn on the device (the cache-length sweep needs no host copies)
+            if not host_copies:
+                # same distribution, drawn on the device
                 gen = torch.Generator(device=dev).manual_seed(cfg.seed * 7919 + l)
                 mk = lambda *sh: (torch.randn(*sh, generator=gen, device=dev, dtype=torch.float32) * cfg.input_scale).to(dt)
                 self.layers.append(dict(
                     kc=mk(Hkv, L + n, D), vc=mk(Hkv, L + n, D), q=mk(n, Hq, D), k=mk(n, Hkv, D), v=mk(n, Hkv, D),
                     q_rot=torch.empty(qbytes, dtype=torch.uint8, device=dev),
-                    ws=torch.empty(wbytes, dtype=torch.uint8, device=dev),
+                    ws=torch.empty(max(wbytes, 16), dtype=torch.uint8, device=dev),
                     out=torch.empty((n, Hq, D), dtype=dt, device=dev)))
                 kc = self.layers[-1]["kc"]
                 continue
@@ -165,16 +173,21 @@ class LayerRing:
             # leaves); the calls take its three strided views
             host_qkv = torch.cat([x["q_new"], x["k_new"], x["v_new"]], dim=1).contiguous().pin_memory()
             qkv = host_qkv.to(dev)
-            host_in = [host_qkv]
             self.layers.append(dict(
                 kc=kc, vc=vc, qkv=qkv, q=qkv[:, :Hq], k=qkv[:, Hq:Hq + Hkv], v=qkv[:, Hq + Hkv:],
                 q_rot=torch.empty(qbytes, dtype=torch.uint8, device=dev),
-                ws=torch.empty(wbytes, dtype=torch.uint8, device=dev),
+                ws=torch.empty(max(wbytes, 16), dtype=torch.uint8, device=dev),
                 out=torch.empty((n, Hq, D), dtype=dt, device=dev),
-                host_in=host_in,
+                host_in=[host_qkv],
                 host_out=torch.empty((n, Hq, D), dtype=dt).pin_memory(),
             ))
         self.bytes_per_layer = 2 * kc.numel() * kc.element_size()
+        self.make_table()
+        torch.cuda.synchronize()
+
+    def make_table(self):
+        c = self.cfg
+        self.B.evlnRopeTable(self.h, c.head_dim, c.rope_theta, c.cache_len, c.num_new, self.table)
 
     def step(self, l):
         B, y = self.B, self.layers[l]
@@ -182,9 +195,17 @@ class LayerRing:
         B.evlnStepAttention(self.h, self.p, y["q_rot"], y["kc"], y["vc"], y["ws"])
         B.evlnStepCombine(self.h, self.p, y["ws"], y["out"], None)
 
+    def append_only(self, l):
+        y = self.layers[l]
+        self.B.evlnRopeAppend(self.h, self.p, y["q"], y["k"], y["v"], y["q_rot"], y["kc"], y["vc"])
+
     def attention_only(self, l):
         y = self.layers[l]
         self.B.evlnStepAttention(self.h, self.p, y["q_rot"], y["kc"], y["vc"], y["ws"])
+
+    def combine_only(self, l):
+        y = self.layers[l]
+        self.B.evlnStepCombine(self.h, self.p, y["ws"], y["out"], None)
 
     def step_e2e(self, l, s_in=None, s_out=None):
         """Host buffers in, host buffer out.  With side streams the host-to-device copies, the
@@ -211,6 +232,7 @@ class LayerRing:
             cur = torch.cuda.current_stream()
             s_in.wait_stream(cur)
             s_out.wait_stream(cur)
+            self.make_table()
             for l in range(len(self.layers)):
                 self.step_e2e(l, s_in, s_out)
             cur.wait_stream(s_in)
@@ -218,33 +240,109 @@ class LayerRing:
         return g
 
 
-def capture(fn, layers):
+class PagedBatch:
+    """The batched-serving workload (16 episodes on a page pool) on the device, one or more
+    independent layers (pools), as CUDA-graph-able calls."""
+
+    def __init__(self, B, handle, cfg, x, dev, layers):
+        self.B, self.h, self.cfg = B, handle, cfg
+        Bn, P, Hq, Hkv, D = len(x["cache_lens"]), cfg.page_size, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
+        self.lens, self.offs = x["cache_lens"], x["new_offsets"]
+        max_pages = max(len(t) for t in x["page_table"])
+        table = torch.zeros((Bn, max_pages), dtype=torch.int32)
+        for b, t in enumerate(x["page_table"]):
+            table[b, :len(t)] = torch.tensor(t, dtype=torch.int32)
+        self.table = table.to(dev)
+        self.p = B.paged_params(Hq, Hkv, D, Bn, P, x["num_pages"], max_pages, cfg.rope_theta)
+        total = self.offs[-1]
+        wbytes = B.evlnPagedWorkspaceSize(handle, self.p, self.lens, self.offs)
+        self.layers = []
+        for l in range(layers):
+            # layer 0 holds the seeded pools; further layers hold independent random pools of the same shape
+            if l == 0:
+                kp = x["k_pool"].to(dev).permute(0, 2, 1, 3).contiguous()
+                vp = x["v_pool"].to(dev).permute(0, 2, 1, 3).contiguous()
+            else:
+                gen = torch.Generator(device=dev).manual_seed(cfg.seed * 7919 + l)
+                mk = lambda *sh: (torch.randn(*sh, generator=gen, device=dev, dtype=torch.float32) * cfg.input_scale).to(torch.bfloat16)
+                kp, vp = mk(x["num_pages"], Hkv, P, D), mk(x["num_pages"], Hkv, P, D)
+            self.layers.append(dict(
+                kp=kp, vp=vp, q=x["q_new"].to(dev), k=x["k_new"].to(dev), v=x["v_new"].to(dev),
+                q_rot=torch.empty(total * Hq * D * 2 + 256, dtype=torch.uint8, device=dev),
+                ws=torch.empty(wbytes, dtype=torch.uint8, device=dev),
+                out=torch.empty((total, Hq, D), dtype=torch.bfloat16, device=dev)))
+        self.kv_bytes = sum(2 * (L + (self.offs[b + 1] - self.offs[b])) * Hkv * D * 2 for b, L in enumerate(self.lens))
+        G = Hq // Hkv
+        self.flops = sum(4 * D * Hq * ((self.offs[b + 1] - self.offs[b]) * L
+                                       + (self.offs[b + 1] - self.offs[b]) * (self.offs[b + 1] - self.offs[b] + 1) // 2)
+                         for b, L in enumerate(self.lens))
+        self.alg_bytes = self.kv_bytes + 2 * total * Hq * D * 2 + 4 * total * Hkv * D * 2
+
+    def step(self, l):
+        B, y = self.B, self.layers[l]
+        B.evlnPagedRopeAppend(self.h, self.p, y["q"], y["k"], y["v"], self.lens, self.offs, self.table, y["q_rot"], y["kp"], y["vp"])
+        B.evlnPagedStepAttention(self.h, self.p, y["q_rot"], y["kp"], y["vp"], self.lens, self.offs, self.table, y["ws"])
+        B.evlnPagedStepCombine(self.h, self.p, y["ws"], self.lens, self.offs, y["out"], None)
+
+    def attention_only(self, l):
+        y = self.layers[l]
+        self.B.evlnPagedStepAttention(self.h, self.p, y["q_rot"], y["kp"], y["vp"], self.lens, self.offs, self.table, y["ws"])
+
+
+def capture(fn, layers, before=None):
     g = torch.cuda.CUDAGraph()
     s = torch.cuda.Stream()
     s.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(s):
+        if before is not None:
+            before()
         for l in range(layers):
             fn(l)                                    # warm the path on the side stream
     torch.cuda.current_stream().wait_stream(s)
     torch.cuda.synchronize()
     with torch.cuda.graph(g):
+        if before is not None:
+            before()
         for l in range(layers):
             fn(l)
     return g
 
 
-def timed(run_chunk, chunks, barrier):
-    """Barrier + sync, CUDA events around `chunks` calls of run_chunk on the current stream."""
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+CLOCKS = None               # the run's ClockSampler: records while a timed region is open
+
+
+def timed_replays(graph, replays, per_replay, barrier, warm=3):
+    """`warm` untimed replays, then barrier + sync, CUDA events around EACH of `replays` replays of the
+    graph on the current stream.  Returns microseconds per unit (a replay holds `per_replay` units):
+    mean over the whole timed region, median / p10 / p90 over the replays."""
+    for _ in range(warm):
+        graph.replay()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(replays + 1)]
     barrier()
     torch.cuda.synchronize()
-    e0.record()
-    for _ in range(chunks):
-        run_chunk()
-    e1.record()
+    if CLOCKS is not None:
+        CLOCKS.recording.set()
+    ev[0].record()
+    for r in range(replays):
+        graph.replay()
+        ev[r + 1].record()
     torch.cuda.synchronize()
+    if CLOCKS is not None:
+        CLOCKS.recording.clear()
     barrier()
-    return e0.elapsed_time(e1)            # ms
+    per = sorted(ev[r].elapsed_time(ev[r + 1]) * 1e3 / per_replay for r in range(replays))
+    pick = lambda q: per[min(len(per) - 1, int(q * len(per)))]
+    return {"mean": ev[0].elapsed_time(ev[replays]) * 1e3 / (replays * per_replay), "median": pick(0.5),
+            "p10": pick(0.1), "p90": pick(0.9), "replays": replays}
+
+
+def r3(x):
+    return round(x, 3)
+
+
+def ring_layers_for(kv_bytes):
+    """Enough independent layers that the K/V revisited round-robin exceed the L2 more than twice."""
+    return max(2, min(RING_LAYERS, int(2.2 * L2_BYTES / kv_bytes) + 1))
 
 
 def run_ours(args, rank, world, local_rank, dist):
@@ -253,11 +351,8 @@ def run_ours(args, rank, world, local_rank, dist):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     cfg = W.STEP_7B
+    peaks, peaks_kind = load_peaks()
     handle = B.evlnCreate(local_rank)
-    ring = LayerRing(B, handle, cfg, dev, RING_LAYERS)
-    for l in range(RING_LAYERS):
-        ring.step(l)
-    assert B.evlnGetDeviceStatus(handle) == 0
 
     def barrier():
         if dist is not None:
@@ -266,128 +361,179 @@ def run_ours(args, rank, world, local_rank, dist):
     def max_over_ranks(x):
         return _max_over_ranks(x, dist, dev)
 
-    steps = max(RING_LAYERS, (args.steps // RING_LAYERS) * RING_LAYERS)
-    warm = max(3 * RING_LAYERS, -(-args.warmup // RING_LAYERS) * RING_LAYERS)
-    g_step = capture(ring.step, RING_LAYERS)
-    g_attn = capture(ring.attention_only, RING_LAYERS)
+    def roof_us(flops, abytes):
+        return max(flops / (peaks["bf16_tflops"] * 1e12), abytes / (peaks["hbm_gbs"] * 1e9)) * 1e6
 
-    for _ in range(warm // RING_LAYERS):
-        g_step.replay()
-    torch.cuda.synchronize()
+    replays = max(MIN_REPLAYS, -(-args.steps // RING_LAYERS))
+    steps = replays * RING_LAYERS
+    warm_replays = max(3, -(-args.warmup // RING_LAYERS))
 
-    sampler = ClockSampler(physical_gpu_index(local_rank))
+    global CLOCKS
+    sampler = CLOCKS = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-    ms = timed(g_step.replay, steps // RING_LAYERS, barrier)
-    ms_attn = timed(g_attn.replay, steps // RING_LAYERS, barrier)
-    clocks = sampler.stop()
+
+    # ---- headline: the 7B-class layer-step (L = 4096, n = 196) ----
+    ring = LayerRing(B, handle, cfg, dev, RING_LAYERS, host_copies=True)
+    for l in range(RING_LAYERS):
+        ring.step(l)
+    assert B.evlnGetDeviceStatus(handle) == 0
+    g_step = capture(ring.step, RING_LAYERS, before=ring.make_table)
+    g_k1 = capture(ring.append_only, RING_LAYERS)
+    g_attn = capture(ring.attention_only, RING_LAYERS)
+    g_k3 = capture(ring.combine_only, RING_LAYERS)
+    t_step = timed_replays(g_step, replays, RING_LAYERS, barrier, warm_replays)
+    t_attn = timed_replays(g_attn, replays, RING_LAYERS, barrier, warm_replays)
+    t_k1 = timed_replays(g_k1, replays, RING_LAYERS, barrier, warm_replays)
+    t_k3 = timed_replays(g_k3, replays, RING_LAYERS, barrier, warm_replays)
     assert B.evlnGetDeviceStatus(handle) == 0, "a kernel gave up on a bounded wait"
 
-    # end to end through the public calls with host buffers (eager launches + copies)
-    e2e_steps = min(steps, 64 * RING_LAYERS)
+    # end to end through the public calls with host buffers
     for l in range(RING_LAYERS):
         ring.step_e2e(l)
     torch.cuda.synchronize()
-
     g_e2e = ring.capture_e2e()
-    for _ in range(3):
-        g_e2e.replay()
-    torch.cuda.synchronize()
-    ms_e2e = timed(g_e2e.replay, e2e_steps // RING_LAYERS, barrier)
+    e2e_replays = min(replays, 400)
+    t_e2e = timed_replays(g_e2e, e2e_replays, RING_LAYERS, barrier, 3)
 
-    us_step = max_over_ranks(ms * 1e3 / steps)
-    us_attn = max_over_ranks(ms_attn * 1e3 / steps)
-    us_e2e = max_over_ranks(ms_e2e * 1e3 / e2e_steps)
-
-    # The metric is quoted against the cache length: the same layer-step at other L (7B-class shape),
-    # a short measurement each, on rank 0 of a single-GPU run only.
+    us_step = max_over_ranks(t_step["mean"])
+    us_attn = max_over_ranks(t_attn["mean"])
+    us_e2e = max_over_ranks(t_e2e["mean"])
     h2d = sum(t.numel() * t.element_size() for t in ring.layers[0]["host_in"])
     d2h = ring.layers[0]["host_out"].numel() * ring.layers[0]["host_out"].element_size()
-    by_len, action_steps = [], []
+    ring_mib = RING_LAYERS * ring.bytes_per_layer / 2 ** 20
+    headline_splits = ring.splits
+
+    by_len, action_steps, by_config = [], [], []
     if world == 1 and not args.no_sweep:
-        del g_step, g_attn
+        del g_step, g_attn, g_k1, g_k3, g_e2e
         ring.layers.clear()
         torch.cuda.empty_cache()
-        peaks_s, _ = load_peaks()
-        for L in (1024, 8192, 16384, 32768):
-            c = dataclasses.replace(cfg, name=f"step_7b_L{L}", cache_len=L)
-            kv_bytes = 2 * (L + c.num_new) * c.num_kv_heads * c.head_dim * 2
-            layers = max(2, min(RING_LAYERS, int(2.2 * L2_BYTES / kv_bytes) + 1))
-            r = LayerRing(B, handle, c, dev, layers, random_device_inputs=True)
-            gs, ga = capture(r.step, layers), capture(r.attention_only, layers)
-            reps = max(3, 640 // layers)
-            for _ in range(3):
-                gs.replay()
-            t_s = timed(gs.replay, reps, barrier) * 1e3 / (reps * layers)
-            t_a = timed(ga.replay, reps, barrier) * 1e3 / (reps * layers)
-            roof = max(c.flops() / (peaks_s["bf16_tflops"] * 1e12), c.algorithmic_bytes() / (peaks_s["hbm_gbs"] * 1e9)) * 1e6
-            by_len.append({"cache_len": L, "us_per_step": round(t_s, 2), "attention_us": round(t_a, 2),
-                           "attention_tflops": round(c.flops() / t_a / 1e6, 1), "kv_splits": r.splits,
-                           "step_roofline_frac": round(roof / t_s, 4)})
+
+        def measure(c, tag):
+            """Step and attention-only time of one contiguous-cache workload (device-resident inputs)."""
+            kv_bytes = 2 * (c.cache_len + c.num_new) * c.num_kv_heads * c.head_dim * 2
+            layers = ring_layers_for(kv_bytes)
+            r = LayerRing(B, handle, c, dev, layers)
+            gs = capture(r.step, layers, before=r.make_table)
+            ga = capture(r.attention_only, layers)
+            reps = max(MIN_REPLAYS, 6400 // layers) if kv_bytes < 64e6 else MIN_REPLAYS
+            ts = timed_replays(gs, reps, layers, barrier)
+            ta = timed_replays(ga, reps, layers, barrier)
+            roof = roof_us(c.flops(), c.algorithmic_bytes())
+            rec = {"workload": tag, "cache_len": c.cache_len, "new_tokens": c.num_new, "kv_splits": r.splits,
+                   "us_per_step": r3(ts["median"]), "us_p10": r3(ts["p10"]), "us_p90": r3(ts["p90"]),
+                   "attention_us": r3(ta["median"]), "attention_us_p10": r3(ta["p10"]), "attention_us_p90": r3(ta["p90"]),
+                   "attention_tflops": round(c.flops() / ta["median"] / 1e6, 1),
+                   "attention_frac_of_peak": round(c.flops() / ta["median"] / 1e6 / peaks["bf16_tflops"], 4),
+                   "roofline_us": r3(roof), "step_roofline_frac": round(roof / ts["median"], 4),
+                   "replays": reps, "ring_layers": layers}
             del gs, ga, r
             torch.cuda.empty_cache()
-        # The 8 action tokens that follow a frame in the streaming episode (same layer shape): a step
-        # bound by streaming K and V once, quoted against the measured HBM bandwidth.
+            return rec, kv_bytes
+
+        # latency against the cache length at the 7B-class shape
+        for L in (1024, 2048, 8192, 16384, 32768):
+            rec, _ = measure(dataclasses.replace(cfg, name=f"step_7b_L{L}", cache_len=L), f"7B shape, L={L}")
+            by_len.append(rec)
+        # the streaming episode: frame steps 1, 25, 50, 100 of 100 (n = 204; per layer of the 28)
+        for s in (1, 25, 50, 100):
+            rec, _ = measure(W.STREAM_7B.step_config(s), f"streaming episode step {s} of 100 (per layer)")
+            by_config.append(rec)
+        # the 70B-class long-history step
+        rec, _ = measure(W.LONG_70B, "70B-class head shape, L=32768, n=256")
+        by_config.append(rec)
+        # the 8 action tokens that follow a frame (same layer shape): bound by streaming K and V once
         for L in (4096, 20656):
             c = dataclasses.replace(cfg, name=f"action_7b_L{L}", cache_len=L, num_new=8)
-            kv_bytes = 2 * (L + c.num_new) * c.num_kv_heads * c.head_dim * 2
-            layers = max(2, min(RING_LAYERS, int(2.2 * L2_BYTES / kv_bytes) + 1))
-            r = LayerRing(B, handle, c, dev, layers, random_device_inputs=True)
-            gs = capture(r.step, layers)
-            reps = max(3, 640 // layers)
-            for _ in range(3):
-                gs.replay()
-            t_s = timed(gs.replay, reps, barrier) * 1e3 / (reps * layers)
-            action_steps.append({"cache_len": L, "new_tokens": 8, "us_per_step": round(t_s, 2), "kv_splits": r.splits,
-                                 "kv_gbs": round(kv_bytes / t_s / 1e3, 1),
-                                 "hbm_frac": round(kv_bytes / t_s / 1e3 / peaks_s["hbm_gbs"], 4)})
-            del gs, r
-            torch.cuda.empty_cache()
+            rec, kv_bytes = measure(c, f"action tokens, L={L}")
+            rec["kv_gbs"] = round(kv_bytes / rec["us_per_step"] / 1e3, 1)
+            rec["hbm_frac"] = round(kv_bytes / rec["us_per_step"] / 1e3 / peaks["hbm_gbs"], 4)
+            action_steps.append(rec)
+        # batched serving on the page pool: 16 episodes, one launch triple per layer
+        pc = W.PAGED_B16
+        x = W.make_paged_inputs(pc)
+        pb = PagedBatch(B, handle, pc, x, dev, layers=2)
+        gs, ga = capture(pb.step, 2), capture(pb.attention_only, 2)
+        ts = timed_replays(gs, MIN_REPLAYS, 2, barrier)
+        ta = timed_replays(ga, MIN_REPLAYS, 2, barrier)
+        roof = roof_us(pb.flops, pb.alg_bytes)
+        rec = {"workload": "paged batch: 16 episodes, 64-token pages, L in [1024, 16384], n=196 each",
+               "us_per_step": r3(ts["median"]), "us_p10": r3(ts["p10"]), "us_p90": r3(ts["p90"]),
+               "attention_us": r3(ta["median"]), "attention_tflops": round(pb.flops / ta["median"] / 1e6, 1),
+               "attention_frac_of_peak": round(pb.flops / ta["median"] / 1e6 / peaks["bf16_tflops"], 4),
+               "flops": pb.flops, "roofline_us": r3(roof), "step_roofline_frac": round(roof / ts["median"], 4),
+               "replays": MIN_REPLAYS, "ring_layers": 2}
+        if not args.no_cpu_baseline:
+            from oracle import step_oracle as so
+            f64 = lambda t: np.ascontiguousarray(t.to(torch.float64).numpy())
+            t0 = time.perf_counter()
+            so.step_paged(f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"]), f64(x["k_pool"]), f64(x["v_pool"]),
+                          x["page_table"], x["cache_lens"], x["new_offsets"], pc.rope_theta, storage="bf16")
+            rec["oracle_s"] = round(time.perf_counter() - t0, 2)
+        by_config.append(rec)
+        del gs, ga, pb, x
+        torch.cuda.empty_cache()
+        if not args.no_cpu_baseline:
+            dt, _ = cpu_baseline_full_step(W.LONG_70B, reps=1)
+            by_config[-2]["oracle_s"] = round(dt, 2)
         assert B.evlnGetDeviceStatus(handle) == 0, "a kernel gave up on a bounded wait"
+    clocks = sampler.stop()
     B.evlnDestroy(handle)
     if rank != 0:
         return None
 
-    peaks, peaks_kind = load_peaks()
     flops = cfg.flops()
     abytes = cfg.algorithmic_bytes()
     t_flop_us = flops / (peaks["bf16_tflops"] * 1e12) * 1e6
     t_hbm_us = abytes / (peaks["hbm_gbs"] * 1e9) * 1e6
     achieved_tf = flops / (us_attn * 1e-6) / 1e12
+    spread = lambda t: {"median": r3(t["median"]), "p10": r3(t["p10"]), "p90": r3(t["p90"]), "mean": r3(t["mean"]),
+                        "replays": t["replays"]}
     line = {
         "metric": "new-frame step-attention latency", "value": round(us_step, 3), "unit": "us/step",
-        "n_gpus": world, "steps": steps, "warmup": warm, "ms_per_step": us_step / 1e3,
+        "n_gpus": world, "steps": steps, "warmup": warm_replays * RING_LAYERS, "ms_per_step": us_step / 1e3,
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {
             "workload": f"{cfg.name}: 28q/4kv heads, head_dim 128, L=4096, n=196, theta 1e6, bf16, one layer-step "
-                        "= evlnRopeAppend + evlnStepAttention + evlnStepCombine",
-            "kv_splits": ring.splits,
-            "launch": f"CUDA graph of {RING_LAYERS} layer-steps, replayed",
+                        "= evlnRopeAppend + evlnStepAttention + evlnStepCombine (position table made once per "
+                        f"{RING_LAYERS} layer-steps by evlnRopeTable)",
+            "kv_splits": headline_splits,
+            "launch": f"CUDA graph of {RING_LAYERS} layer-steps, replayed {replays} times (at least {MIN_REPLAYS} "
+                      "whatever --steps asks for), CUDA events around every replay",
             "l2": f"inputs larger than L2: ring of {RING_LAYERS} independent layer caches, "
-                  f"{RING_LAYERS * ring.bytes_per_layer / 2**20:.0f} MiB of K/V revisited round-robin",
+                  f"{ring_mib:.0f} MiB of K/V revisited round-robin",
             "parallelism": "replicas only" if world > 1 else "single GPU",
         },
+        "us_per_step": spread(t_step),
+        "kernels_us": {"rope_append": spread(t_k1), "attention": spread(t_attn), "combine": spread(t_k3)},
         "tflops": round(flops / (us_step * 1e-6) / 1e12 * world, 2),
         "gbs": round(abytes / (us_step * 1e-6) / 1e9 * world, 1),
         "steps_per_s": round(aggregate_steps_per_s(us_step, world), 1),
+        "roofline_us": r3(max(t_flop_us, t_hbm_us)),
         "step_roofline_frac": round(max(t_flop_us, t_hbm_us) / us_step, 4),
         "roofline": {
             "kernel": "attn_pair_kernel (evlnStepAttention)", "bound": "tensor",
             "achieved": round(achieved_tf, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
             "frac": round(achieved_tf / peaks["bf16_tflops"], 4), "peak_kind": f"{peaks_kind} burst bf16",
+            "frac_of_sustained": round(achieved_tf / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), 4),
             "traffic": attention_dram_traffic(), "us_per_launch": round(us_attn, 3),
-            "timing": f"CUDA events around graph replays of {RING_LAYERS} back-to-back attention launches",
+            "us_per_launch_median": r3(t_attn["median"]), "us_per_launch_p10": r3(t_attn["p10"]),
+            "us_per_launch_p90": r3(t_attn["p90"]),
+            "timing": f"CUDA events around each of {replays} graph replays of {RING_LAYERS} back-to-back attention launches",
             "flops_per_launch": flops,
         },
         "e2e": {"value": round(us_e2e, 3), "unit": "us/step", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "d2h_bytes_per_step": d2h, "steps": e2e_replays * RING_LAYERS, "median": r3(t_e2e["median"]),
                 "launch": f"CUDA graph of {RING_LAYERS} steps: pinned host-to-device copies, the three calls, "
                           "device-to-host copy; copies on side streams overlap the neighbouring steps' kernels"},
-        "gpu_launches": 3 * steps,
+        "gpu_launches": (3 * RING_LAYERS + 1) * replays,
         "clocks": clocks,
     }
     if by_len:
         line["by_cache_len"] = by_len
+    if by_config:
+        line["by_config"] = by_config
     if action_steps:
         line["action_token_step"] = action_steps
     return line
@@ -421,8 +567,8 @@ def oracle_sample_time(cfg, tokens_per_step, steps, warmup):
     return total / steps, so.num_threads()
 
 
-def cpu_baseline_full_step(cfg):
-    """One full step of the oracle (all query rows), threads as the oracle uses them."""
+def cpu_baseline_full_step(cfg, reps=5):
+    """Full steps of the oracle (all query rows), threads as the oracle uses them."""
     from oracle import step_oracle as so
     x = W.make_step_inputs(cfg)
     f64 = lambda t: np.ascontiguousarray(t.to(torch.float64).numpy())
@@ -431,7 +577,6 @@ def cpu_baseline_full_step(cfg):
     vc = np.zeros_like(kc)
     kc[:L], vc[:L] = f64(x["k_cache"]), f64(x["v_cache"])
     q, k, v = f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"])
-    reps = 5
     t0 = time.perf_counter()
     for _ in range(reps):
         so.step(q, k, v, kc, vc, L, cfg.rope_theta, storage="bf16")
@@ -475,11 +620,11 @@ def run_reference(args, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=65536)
-    ap.add_argument("--warmup", type=int, default=3200)
+    ap.add_argument("--steps", type=int, default=32768)
+    ap.add_argument("--warmup", type=int, default=640)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the short cache-length sweep")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads (cache-length sweep, by_config)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))

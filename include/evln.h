@@ -81,6 +81,13 @@ typedef struct {
     int kernel;              /* evlnKernel_t                                                 */
     float softmax_scale;     /* 0 -> 1/sqrt(D)                                               */
     double rope_theta;       /* RoPE base, > 0                                               */
+    /* Optional position table written by evlnRopeTable (NULL: the kernels form the angles
+     * themselves, once per call).  It must cover positions L .. L+n-1, i.e.
+     * rope_table_first_pos <= L and L+n <= rope_table_first_pos + rope_table_count, and must
+     * have been made for this head_dim and rope_theta.  Results are bit-identical either way. */
+    const void* rope_table;
+    int rope_table_first_pos;
+    int rope_table_count;
 } evlnStepParams;
 
 /* A batch of episodes on a page pool (one layer).  Episode b has h_cache_lens[b] cached
@@ -103,7 +110,9 @@ typedef struct {
 /* ---- handle, errors ------------------------------------------------------------------- */
 
 /* Creates a handle bound to CUDA device `device` (allocates a 4-byte device status word and
- * resolves the driver's tensor-map encoder).  Sec. 3.2 has no counterpart: plumbing.        */
+ * resolves the driver's tensor-map encoder); the caller's current device is left as it was.
+ * Every call that launches work must be made with that device current, otherwise it returns
+ * EVLN_INVALID_VALUE and launches nothing.  Sec. 3.2 has no counterpart: plumbing.          */
 evlnStatus_t evlnCreate(evlnHandle_t* handle, int device);
 evlnStatus_t evlnDestroy(evlnHandle_t handle);
 const char* evlnGetErrorString(evlnStatus_t status);
@@ -111,8 +120,19 @@ const char* evlnGetErrorString(evlnStatus_t status);
 int evlnGetLastCudaError(evlnHandle_t handle);
 /* Synchronises `stream`, reads and clears the device status word.  *device_status = 0 when no
  * kernel gave up on a bounded wait; otherwise a code identifying the wait that expired and
- * the function returns EVLN_DEVICE_TIMEOUT (the outputs of that step are then invalid).     */
+ * the function returns EVLN_DEVICE_TIMEOUT (the outputs of that step are then invalid).
+ * handle == NULL addresses the status word of the allocation-free call
+ * (evlnStepAttentionNoAlloc) on the CURRENT device; it allocates nothing either.             */
 evlnStatus_t evlnGetDeviceStatus(evlnHandle_t handle, void* stream, int* device_status);
+
+/* Self-test of the fault containment (Sec. 3.2 has no counterpart: plumbing).  Launches one
+ * small kernel whose only act is a bounded wait on a barrier that nothing ever arrives on, with
+ * a limit of `limit_cycles` SM clocks (1000 .. 10^9): the wait must run out, the kernel must
+ * record EVLN_SELFTEST_STATUS_CODE in the handle's status word and return normally, so that the
+ * next evlnGetDeviceStatus reports EVLN_DEVICE_TIMEOUT with that code and the context stays
+ * usable.  No fault, trap or unbounded loop is involved.                                     */
+#define EVLN_SELFTEST_STATUS_CODE 8
+evlnStatus_t evlnSelfTestBoundedWait(evlnHandle_t handle, long long limit_cycles, void* stream);
 
 /* ---- contiguous cache ------------------------------------------------------------------- */
 
@@ -123,6 +143,17 @@ evlnStatus_t evlnStepNumSplits(evlnHandle_t handle, const evlnStepParams* params
 evlnStatus_t evlnStepWorkspaceSize(evlnHandle_t handle, const evlnStepParams* params, size_t* bytes);
 /* Bytes of the q_rot scratch: n * Hq * D elements, rounded up to 256. */
 evlnStatus_t evlnStepQRotSize(evlnHandle_t handle, const evlnStepParams* params, size_t* bytes);
+
+/* RoPE position table (Sec. 3.2: one set of contiguous position ids per navigation step, shared
+ * by all layers).  Entry (p, j), p = 0 .. count-1, j = 0 .. head_dim/2-1, holds the pair
+ * (cos, sin) of (first_pos + p) * rope_theta^(-2j/head_dim) as two doubles: exactly the values
+ * evlnRopeAppend / evlnGatherRope would form themselves in every call.  The angles depend on the
+ * position only, so a model computes the table once per step and passes it to the calls of all
+ * its layers (evlnStepParams.rope_table, evlnGatherParams.rope_table).
+ * evlnRopeTableBytes = count * (head_dim/2) * 16; `table` must be 16-byte aligned device memory. */
+size_t evlnRopeTableBytes(int head_dim, int count);
+evlnStatus_t evlnRopeTable(evlnHandle_t handle, int head_dim, double rope_theta, int first_pos,
+                           int count, void* table, void* stream);
 
 /* Step 1 (Sec. 3.2: contiguous position ids, RoPE, concatenation with the cache).
  * Rotates the new queries at positions L+i into q_rot (grouped by kv head), rotates the new
@@ -186,6 +217,16 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t handle, const evlnPagedParams* pa
                                   const void* workspace, const int* h_cache_lens,
                                   const int* h_new_offsets, void* out, float* lse_out,
                                   void* stream);
+/* Host-side check of a page table BEFORE it is copied to the device (no GPU work; plumbing).
+ * h_page_table is the host copy, int [batch, max_pages_per_seq].  For every episode the first
+ * ceil((L_b + n_b) / page_size) entries must be pool pages in [0, num_pages) and no page may be
+ * listed twice, by one episode or by two: the append kernel writes through this table, so a bad
+ * entry would corrupt another episode's cache or write outside the pool.  Returns EVLN_OK,
+ * EVLN_INVALID_VALUE (bad entry; *h_bad_episode / *h_bad_index, if not NULL, say where) or the
+ * usual parameter errors.                                                                    */
+evlnStatus_t evlnPagedCheckTable(const evlnPagedParams* params, const int* h_cache_lens,
+                                 const int* h_new_offsets, const int* h_page_table,
+                                 int* h_bad_episode, int* h_bad_index);
 
 /* ---- allocation-free variant ------------------------------------------------------------ */
 
@@ -211,7 +252,11 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t handle, const evlnPagedParams* pa
  *
  * Set-up: the first call on each device (with that device current) looks up the scratch
  * array's device address and the device's properties once; make that first call outside any
- * stream capture.  Later calls on that device only validate and launch.
+ * stream capture.  Later calls on that device only validate and launch.  Host threads may race
+ * for the first call: the set-up runs once per device under a lock.
+ * Status: a kernel of this call that gives up on a bounded wait records it in a status word
+ * that is part of the library image as well; evlnGetDeviceStatus(NULL, stream, &code) reads and
+ * clears it for the current device.
  * Limits and errors: parameters whose split workspace (evlnStepWorkspaceSize) exceeds
  * EVLN_NOALLOC_SCRATCH_BYTES are rejected with EVLN_WORKSPACE_TOO_SMALL and nothing is
  * launched; other errors as for evlnStepAttention / evlnStepCombine.
@@ -223,8 +268,8 @@ evlnStatus_t evlnStepAttentionNoAlloc(const evlnStepParams* params, const void* 
                                       const void* k_cache, const void* v_cache, void* out,
                                       float* lse_out, void* stream);
 
-/* ---- un-rotated store + frame sampler (Sec. 3.2, "store the KV cache prior to the rotation",
- *      frame samplers "uniform" and "sliding window") -------------------------------------
+/* ---- un-rotated store + frame sampler (Sec. 3.2: the cache is kept un-rotated; kept tokens are
+ *      re-rotated at contiguous ids; uniform and sliding-window frame samplers) -----------
  *
  * The episode's raw keys and values (as projected, NOT rotated) live in a store
  * [Hkv, store_capacity, D] per layer.  Every step the caller
@@ -244,6 +289,10 @@ typedef struct {
     int store_capacity;      /* token slots per kv head in k_store / v_store                 */
     int work_capacity;       /* token slots per kv head in k_work / v_work                   */
     double rope_theta;
+    /* optional evlnRopeTable table covering the positions 0 .. (tokens laid out)-1 (NULL: none) */
+    const void* rope_table;
+    int rope_table_first_pos;
+    int rope_table_count;
 } evlnGatherParams;
 
 typedef enum { EVLN_SAMPLE_UNIFORM = 0, EVLN_SAMPLE_SLIDING = 1 } evlnSampler_t;
@@ -274,8 +323,8 @@ evlnStatus_t evlnGatherRope(evlnHandle_t handle, const evlnGatherParams* params,
                             const void* v_store, void* k_work, void* v_work, int* h_total,
                             void* stream);
 
-/* ---- host-resident store (Sec. 3.2, "Memory Management": the cache is offloaded to the CPU and
- *      only the segments the sampler selects are reloaded) ------------------------------------
+/* ---- host-resident store (Sec. 3.2, memory management: the cache lives in host memory and only
+ *      the segments the sampler keeps come back to the GPU) -----------------------------------
  *
  * The full raw store of an episode may live in PINNED host memory, [Hkv, host_capacity, D],
  * while the device store only has room for the segments in use.  evlnStoreOffload copies token

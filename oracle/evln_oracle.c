@@ -5,14 +5,14 @@
  * navigation step computes, written out with ordinary loops in double precision:
  *
  *   1. the new frame's tokens get the position ids that continue the cached
- *      sequence, pos_i = L + i                      (Sec. 3.2, "contiguous position IDs");
+ *      sequence, pos_i = L + i                      (Sec. 3.2: ids stay contiguous);
  *   2. the new queries and keys are rotated by RoPE at those positions
- *      (Sec. 3.2, "apply the RoPE transformation"; 1-D NeoX half-split pairing);
+ *      (Sec. 3.2: rotation applied when the step runs; 1-D NeoX half-split pairing);
  *   3. rotated keys and the unchanged values are appended to the reused cache
- *      (Sec. 3.2, cached tensors "concatenated with the newly encoded frame");
+ *      (Sec. 3.2: the cached tensors are joined with the new frame's);
  *   4. only the new frame is prefilled: each new query attends causally to all
- *      cached tokens and to the new tokens up to itself (Sec. 3.2, "process only the
- *      current frame for ... transformer prefilling").
+ *      cached tokens and to the new tokens up to itself (Sec. 3.2: the transformer
+ *      prefill covers the current frame alone).
  *
  * It shares nothing with the CUDA library: no headers, no constants, no helpers.
  * Only tests, the smoke check and the benchmark's cpu_baseline leg may call it.

@@ -25,20 +25,25 @@ EVLN_KERNEL_AUTO, EVLN_KERNEL_SIMT = 0, 1
 
 EXPORTS = [
     "evlnCreate", "evlnDestroy", "evlnGetErrorString", "evlnGetLastCudaError", "evlnGetDeviceStatus",
+    "evlnSelfTestBoundedWait",
     "evlnStepNumSplits", "evlnStepWorkspaceSize", "evlnStepQRotSize",
+    "evlnRopeTableBytes", "evlnRopeTable",
     "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine", "evlnStep",
     "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
+    "evlnPagedCheckTable",
     "evlnStepAttentionNoAlloc",
     "evlnSampleFrames", "evlnStoreAppend", "evlnGatherRope", "evlnStoreOffload", "evlnStoreFetch",
 ]
 EVLN_NOALLOC_SCRATCH_BYTES = 32 << 20
+EVLN_SELFTEST_STATUS_CODE = 8
 
 
 class evlnStepParams(Structure):
     _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_q_heads", c_int),
                 ("num_kv_heads", c_int), ("head_dim", c_int), ("cache_len", c_int),
                 ("num_new", c_int), ("cache_capacity", c_int), ("num_splits", c_int),
-                ("kernel", c_int), ("softmax_scale", c_float), ("rope_theta", c_double)]
+                ("kernel", c_int), ("softmax_scale", c_float), ("rope_theta", c_double),
+                ("rope_table", c_void_p), ("rope_table_first_pos", c_int), ("rope_table_count", c_int)]
 
 
 class evlnPagedParams(Structure):
@@ -50,7 +55,8 @@ class evlnPagedParams(Structure):
 
 class evlnGatherParams(Structure):
     _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_kv_heads", c_int), ("head_dim", c_int),
-                ("store_capacity", c_int), ("work_capacity", c_int), ("rope_theta", c_double)]
+                ("store_capacity", c_int), ("work_capacity", c_int), ("rope_theta", c_double),
+                ("rope_table", c_void_p), ("rope_table_first_pos", c_int), ("rope_table_count", c_int)]
 
 
 EVLN_SAMPLE_UNIFORM, EVLN_SAMPLE_SLIDING = 0, 1
@@ -97,6 +103,10 @@ def lib():
         L.evlnDestroy.argtypes = [c_void_p]
         L.evlnGetLastCudaError.argtypes = [c_void_p]
         L.evlnGetDeviceStatus.argtypes = [c_void_p, c_void_p, POINTER(c_int)]
+        L.evlnSelfTestBoundedWait.argtypes = [c_void_p, ctypes.c_longlong, c_void_p]
+        L.evlnRopeTableBytes.argtypes = [c_int, c_int]
+        L.evlnRopeTableBytes.restype = c_size_t
+        L.evlnRopeTable.argtypes = [c_void_p, c_int, c_double, c_int, c_int, c_void_p, c_void_p]
         pp = POINTER(evlnStepParams)
         L.evlnStepNumSplits.argtypes = [c_void_p, pp, POINTER(c_int)]
         L.evlnStepWorkspaceSize.argtypes = [c_void_p, pp, POINTER(c_size_t)]
@@ -116,6 +126,7 @@ def lib():
         L.evlnPagedStepAttention.argtypes = [c_void_p, gp, c_void_p, c_void_p, c_void_p, ip, ip, c_void_p,
                                              c_void_p, c_size_t, c_void_p]
         L.evlnPagedStepCombine.argtypes = [c_void_p, gp, c_void_p, ip, ip, c_void_p, c_void_p, c_void_p]
+        L.evlnPagedCheckTable.argtypes = [gp, ip, ip, ip, ip, ip]
         L.evlnStepAttentionNoAlloc.argtypes = [pp, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         qp = POINTER(evlnGatherParams)
         L.evlnSampleFrames.argtypes = [c_int, c_int, c_int, c_int, POINTER(c_int)]
@@ -128,7 +139,7 @@ def lib():
         L.evlnStoreFetch.argtypes = [c_void_p, qp, c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_int,
                                      c_void_p]
         for name in EXPORTS:
-            if name != "evlnGetErrorString":
+            if name not in ("evlnGetErrorString", "evlnRopeTableBytes"):
                 getattr(L, name).restype = c_int
         _lib = L
     return _lib
@@ -167,10 +178,13 @@ def _ints(seq):
 
 
 def step_params(dtype, num_q_heads, num_kv_heads, head_dim, cache_len, num_new, cache_capacity,
-                rope_theta, softmax_scale=0.0, num_splits=0, kernel=EVLN_KERNEL_AUTO) -> evlnStepParams:
+                rope_theta, softmax_scale=0.0, num_splits=0, kernel=EVLN_KERNEL_AUTO,
+                rope_table=None, rope_table_first_pos=0, rope_table_count=0) -> evlnStepParams:
+    """``rope_table``: a tensor written by evlnRopeTable (or None) covering the step's positions."""
     code = {"bf16": EVLN_BF16, "f32": EVLN_F32}.get(dtype, dtype)
     return evlnStepParams(ctypes.sizeof(evlnStepParams), code, num_q_heads, num_kv_heads, head_dim,
-                          cache_len, num_new, cache_capacity, num_splits, kernel, softmax_scale, rope_theta)
+                          cache_len, num_new, cache_capacity, num_splits, kernel, softmax_scale, rope_theta,
+                          _ptr(rope_table), rope_table_first_pos, rope_table_count)
 
 
 def paged_params(num_q_heads, num_kv_heads, head_dim, batch, page_size, num_pages, max_pages_per_seq,
@@ -197,12 +211,37 @@ def evlnGetLastCudaError(handle) -> int:
 
 
 def evlnGetDeviceStatus(handle, stream=None) -> int:
-    """Synchronises the stream; returns the device status word (0 = no bounded wait expired)."""
+    """Synchronises the stream; returns the device status word (0 = no bounded wait expired).
+    ``handle=None`` reads the status word of the allocation-free call on the current device."""
     v = c_int(0)
     st = lib().evlnGetDeviceStatus(handle, _stream(stream), byref(v))
     if st not in (EVLN_OK, EVLN_DEVICE_TIMEOUT):
         raise EvlnError(st, "evlnGetDeviceStatus")
     return int(v.value)
+
+
+def evlnSelfTestBoundedWait(handle, limit_cycles: int = 100000, stream=None):
+    """Launches the self-test kernel whose bounded wait must run out (see include/evln.h)."""
+    _check(lib().evlnSelfTestBoundedWait(handle, int(limit_cycles), _stream(stream)), "evlnSelfTestBoundedWait")
+
+
+def evlnRopeTableBytes(head_dim: int, count: int) -> int:
+    return int(lib().evlnRopeTableBytes(int(head_dim), int(count)))
+
+
+def evlnRopeTable(handle, head_dim, rope_theta, first_pos, count, table, stream=None):
+    """(cos, sin) of the positions first_pos .. first_pos+count-1 into ``table`` (device memory)."""
+    _check(lib().evlnRopeTable(handle, int(head_dim), float(rope_theta), int(first_pos), int(count), _ptr(table),
+                               _stream(stream)), "evlnRopeTable")
+
+
+def evlnPagedCheckTable(params, cache_lens, new_offsets, page_table_rows):
+    """Host check of a page table given as ``[batch][max_pages_per_seq]`` ints (flattened or nested).
+    Returns (status, bad_episode, bad_index)."""
+    flat = [int(v) for row in page_table_rows for v in (row if hasattr(row, "__iter__") else [row])]
+    be, bi = c_int(-1), c_int(-1)
+    st = lib().evlnPagedCheckTable(byref(params), _ints(cache_lens), _ints(new_offsets), _ints(flat), byref(be), byref(bi))
+    return int(st), int(be.value), int(bi.value)
 
 
 def evlnStepNumSplits(handle, params) -> int:
@@ -301,10 +340,11 @@ def evlnStepAttentionNoAlloc(params, q_rot, k_cache, v_cache, out, lse_out=None,
            "evlnStepAttentionNoAlloc")
 
 
-def gather_params(dtype, num_kv_heads, head_dim, store_capacity, work_capacity, rope_theta) -> evlnGatherParams:
+def gather_params(dtype, num_kv_heads, head_dim, store_capacity, work_capacity, rope_theta,
+                  rope_table=None, rope_table_first_pos=0, rope_table_count=0) -> evlnGatherParams:
     code = {"bf16": EVLN_BF16, "f32": EVLN_F32}.get(dtype, dtype)
     return evlnGatherParams(ctypes.sizeof(evlnGatherParams), code, num_kv_heads, head_dim, store_capacity,
-                            work_capacity, rope_theta)
+                            work_capacity, rope_theta, _ptr(rope_table), rope_table_first_pos, rope_table_count)
 
 
 def evlnSampleFrames(sampler: int, num_frames: int, budget: int, stride: int = 1):

@@ -140,7 +140,7 @@ __device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_byte
 }
 
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, int code, int* status,
-                                             volatile int* s_abort)
+                                             volatile int* s_abort, long long limit_cycles = kWaitLimitCycles)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -148,7 +148,7 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, int 
     while (!ptx::mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3f) == 0) {
             if (*s_abort) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *s_abort = 1;
                 atomicCAS(status, 0, code);
                 return false;
@@ -218,14 +218,15 @@ struct WorkItem {
 
 // Contiguous cache: the grid is (CTAS * units, kv heads, splits), so a CTA reads its work item off
 // its block index; the two divisions left (by G and by the split count) are multiplications by
-// constants the host prepared.  Paged batch: items are numbered episode by episode (kv head, unit,
-// split inside), the host passes the first item of every episode and the CTA searches that table.
-template <bool PAGED, typename LensT, int CTAS>
+// constants the host prepared.  Batches (paged cache, or episodes sharing a cache prefix): items are
+// numbered episode by episode (kv head, unit, split inside), the host passes the first item of every
+// episode and the CTA searches that table.
+template <bool PAGED, bool TAIL, typename LensT, int CTAS>
 __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT& lens)
 {
     constexpr int UNIT_ROWS = CTAS * kTileM;
     WorkItem w;
-    if (!PAGED) {
+    if (!PAGED && !TAIL) {
         w.b = 0;
         w.unit = CTAS == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
         w.g = (int)blockIdx.y;
@@ -257,7 +258,8 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
         rem -= w.g * per_head;
         const int units = ceil_div(w.n * a.G, UNIT_ROWS);
         for (int u = 0; u < units; ++u) {
-            const int nkv = unit_kv_tiles_fast(w.L, w.n, a.div_g, u, UNIT_ROWS);
+            const int nkv = TAIL ? tail_kv_tiles_fast(w.L, w.n, a.div_g, u, UNIT_ROWS)
+                                 : unit_kv_tiles_fast(w.L, w.n, a.div_g, u, UNIT_ROWS);
             const int S = ceil_div(nkv, a.chunk_tiles);
             if (rem < S) {
                 w.unit = u;
@@ -276,11 +278,17 @@ __device__ __forceinline__ WorkItem decode_work(const TcAttnArgs& a, const LensT
 // CTAS = 2: launched with a cluster of 2 CTAs along x: query tile = cluster rank.
 // CTAS = 1: no cluster; one query tile (all the rows of a kv head fit in it).
 
-template <bool PAGED, typename LensT, int CTAS>
+// TAIL: a batch of items that share the first L_b tokens of ONE contiguous cache (every row sees all
+// of them) and bring their own n_b new tokens in a separate buffer (tm_kt / tm_vt, packed over the
+// batch; causal among themselves): the action chunks of a packed sequence (Sec. 3.3), each after
+// its own prefix of the visual tokens, none visible to another.
+template <bool PAGED, bool TAIL, typename LensT, int CTAS>
 __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                             const CUtensorMap* tm_kt, const CUtensorMap* tm_vt,
                                              const TcAttnArgs& a, const LensT& lens)
 {
-    static_assert(CTAS == 2 || !PAGED, "the paged kernel runs on CTA pairs");
+    static_assert(CTAS == 2 || !(PAGED || TAIL), "the batch kernels run on CTA pairs");
+    static_assert(!(PAGED && TAIL), "one cache layout at a time");
     using Plan = SmemPlan<CTAS>;
     constexpr int kKStages = Plan::kKStages, kVStages = Plan::kVStages, kStageBytes = Plan::kStageBytes;
     constexpr int kSmemQOff = Plan::kQOff, kSmemKOff = Plan::kKOff, kSmemVOff = Plan::kVOff;
@@ -323,12 +331,13 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
     const uint32_t rank = CTAS == 2 ? ptx::cluster_ctarank() : 0u;   // 0: issues the MMAs, owns the "(CTA 0)" barriers
     if (threadIdx.x == 0) EVLN_STAMP(0);
 
-    const WorkItem w = decode_work<PAGED, LensT, CTAS>(a, lens);
-    if (PAGED && w.b < 0) return;                      // both CTAs of the pair decode the same item
+    const WorkItem w = decode_work<PAGED, TAIL, LensT, CTAS>(a, lens);
+    if ((PAGED || TAIL) && w.b < 0) return;                      // both CTAs of the pair decode the same item
 
     const int rows_valid = w.n * a.G;                            // packed rows of this episode
     const int row0 = w.unit * kItemRows + (int)rank * kTileM;    // first row of this CTA's tile (episode-local)
     const int ntiles = w.j1 - w.j0;
+    const int nct = TAIL ? (w.L + kTileN - 1) / kTileN : 0;      // TAIL: tiles below nct come from the shared cache
     // Lane quarters (32 rows each) of the tile that hold rows of the episode.  A CTA on its own lets
     // the softmax warps of the others sit out; a pair keeps all of them (both CTAs count alike).
     int quarters = 4;
@@ -357,7 +366,11 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         ptx::prefetch_tensormap(&tm_q);
         ptx::prefetch_tensormap(&tm_k);
         ptx::prefetch_tensormap(&tm_v);
-        if (!PAGED) {
+        if (TAIL) {
+            ptx::prefetch_tensormap(tm_kt);
+            ptx::prefetch_tensormap(tm_vt);
+        }
+        if (!PAGED && !TAIL) {
             // this CTA's halves of the first K tiles and of the first V tile on their way into L2 while
             // the pair sets up (cached rows; a row the previous kernel is still writing stays coherent)
             const int pre = ntiles < 3 ? ntiles : 3;
@@ -445,7 +458,15 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 const uint32_t bar = on_cta0(bar_k_full + 8 * stage);
                 const int j = w.j0 + jj;
                 expect(bar, kStageBytes);
-                if (!PAGED) {
+                if (TAIL) {
+                    // shared cache below tile nct (rows past L_b are other items' tokens: finite, masked),
+                    // this item's own tokens after (rows past n_b: the next item's or zero fill, masked)
+                    const bool own = j >= nct;
+                    const int key0 = (own ? lens.new_off[w.b] + (j - nct) * kTileN : j * kTileN) + (int)rank * 64;
+                    const CUtensorMap* map = own ? tm_kt : &tm_k;
+                    tma3(dst, map, bar, 0, key0, w.g);
+                    tma3(dst + kStageBytes / 2, map, bar, 64, key0, w.g);
+                } else if (!PAGED) {
                     const int key0 = j * kTileN + (int)rank * 64;
                     tma3(dst, &tm_k, bar, 0, key0, w.g);
                     tma3(dst + kStageBytes / 2, &tm_k, bar, 64, key0, w.g);
@@ -470,7 +491,11 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 const uint32_t bar = on_cta0(bar_v_full + 8 * stage);
                 const int j = w.j0 + jj;
                 expect(bar, kStageBytes);
-                if (!PAGED) {
+                if (TAIL) {
+                    const bool own = j >= nct;
+                    tma3(dst, own ? tm_vt : &tm_v, bar, 64 * (int)rank,
+                         own ? lens.new_off[w.b] + (j - nct) * kTileN : j * kTileN, w.g);
+                } else if (!PAGED) {
                     tma3(dst, &tm_v, bar, 64 * (int)rank, j * kTileN, w.g);
                     if (CTAS == 1) tma3(dst + kHalfBytes, &tm_v, bar, 64, j * kTileN, w.g);
                 } else {
@@ -592,7 +617,8 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         // last visible key index; a padding row (beyond the episode's rows: its Q is zero fill or
         // another episode's) is never stored, so it takes everything unmasked rather than making its
         // warp mask every tile
-        const int bound = row_valid ? w.L + (int)fast_div((uint32_t)r_local, a.div_g) : 0x3fffffff;
+        // (TAIL: `bound` is the row's last visible token among the item's OWN tokens)
+        const int bound = row_valid ? (TAIL ? 0 : w.L) + (int)fast_div((uint32_t)r_local, a.div_g) : 0x3fffffff;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter << 5) << 16);
         const uint32_t t_s = t_lane + (uint32_t)grp * 128 + (uint32_t)half * 64;          // its half of the group's score buffer
         const uint32_t t_p = t_lane + kColP + (uint32_t)grp * 64 + (uint32_t)half * 32;   // ... and of its P buffer
@@ -757,7 +783,12 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                 if (CTAS == 2) ptx::mbar_arrive_cluster(s_free0); else ptx::mbar_arrive(s_free0);
             }
 
-            const int lim = bound - (w.j0 + jj) * kTileN - half * 64;   // columns 0..lim of this thread's 64 are visible
+            // columns 0..lim of this thread's 64 are visible
+            int lim = bound - (w.j0 + jj) * kTileN - half * 64;
+            if (TAIL) {
+                const int j = w.j0 + jj;
+                lim = (j < nct ? w.L - 1 - j * kTileN : bound - (j - nct) * kTileN) - half * 64;
+            }
             if (!__all_sync(0xffffffffu, lim >= 63)) {
 #pragma unroll
                 for (int blk = 0; blk < 2; ++blk) mask32(&s[blk * 32], lim - blk * 32);   // -inf: masked keys (and stale slots) drop out
@@ -920,7 +951,18 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                  const __grid_constant__ CUtensorMap tm_v, const TcAttnArgs a,
                  const __grid_constant__ LensT lens)
 {
-    attn_tc_body<PAGED, LensT, 2>(tm_q, tm_k, tm_v, a, lens);
+    attn_tc_body<PAGED, false, LensT, 2>(tm_q, tm_k, tm_v, nullptr, nullptr, a, lens);
+}
+
+// CTA pairs over a batch of items that share a prefix of one contiguous cache and bring their own
+// new tokens in a separate buffer (the action chunks of a packed sequence, Sec. 3.3).
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_tail_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kt,
+                 const __grid_constant__ CUtensorMap tm_vt, const TcAttnArgs a,
+                 const __grid_constant__ BatchLens lens)
+{
+    attn_tc_body<false, true, BatchLens, 2>(tm_q, tm_k, tm_v, &tm_kt, &tm_vt, a, lens);
 }
 
 // One CTA per work item, for steps whose rows per kv head fit one 128-row tile (the few action
@@ -930,7 +972,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 attn_solo_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const TcAttnArgs a)
 {
-    attn_tc_body<false, NoLens, 1>(tm_q, tm_k, tm_v, a, NoLens{});
+    attn_tc_body<false, false, NoLens, 1>(tm_q, tm_k, tm_v, nullptr, nullptr, a, NoLens{});
 }
 
 }  // namespace evln

@@ -20,8 +20,10 @@ struct CombineArgs {
     int Hkv, G, D;
     int rows;                // R = (total) new tokens * G
     int num_splits;          // contiguous: S for every row
-    // paged: per-episode split counts are derived from the lengths
+    // batches: per-episode split counts are derived from the lengths
     int batch, unit_rows, chunk_tiles;
+    int tail;                // batch of items sharing a cache prefix (own tokens tiled separately)
+    PackedMap map;           // where output token m goes (identity unless the call serves a packed sequence)
 };
 
 template <typename T, int D, bool PAGED, typename LensT>
@@ -48,7 +50,8 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
         const int n_b = lens.new_off[b + 1] - lens.new_off[b];
         const int local_row = (int)(row - (long)lens.new_off[b] * a.G);
         const int unit = local_row / a.unit_rows;
-        S = ceil_div(unit_kv_tiles(lens.cache_len[b], n_b, a.G, unit, a.unit_rows), a.chunk_tiles);
+        S = ceil_div(a.tail ? tail_kv_tiles(lens.cache_len[b], n_b, a.G, unit, a.unit_rows)
+                            : unit_kv_tiles(lens.cache_len[b], n_b, a.G, unit, a.unit_rows), a.chunk_tiles);
     }
 
     const long stride_s = (long)a.Hkv * a.rows;           // rows between consecutive splits
@@ -124,7 +127,7 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
     }
     const float inv = (wsum > 0.f) ? 1.f / wsum : 0.f;
 
-    const long tok = row / a.G;
+    const long tok = packed_row(a.map, row / a.G);
     const int h = g * a.G + (int)(row % a.G);
     const int Hq = a.Hkv * a.G;
     T* dst = (T*)a.out + (tok * Hq + h) * D + lane * C;

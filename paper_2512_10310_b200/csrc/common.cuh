@@ -24,6 +24,7 @@ enum DeviceStatus : int {
     kDevTimeoutSoftmaxS = 5,   // softmax warps waiting for S
     kDevTimeoutSoftmaxO = 6,   // softmax warps waiting for the final O
     kDevTimeoutSoftmaxX = 7,   // softmax warps of one lane quarter waiting for each other
+    kDevTimeoutSelfTest = 8,   // the self-test's wait on a barrier nothing arrives on (EVLN_SELFTEST_STATUS_CODE)
 };
 
 // Per-episode lengths of a paged batch, passed by value.
@@ -82,6 +83,38 @@ __host__ __device__ inline int unit_kv_tiles_fast(int L, int n, FastDiv div_g, i
     uint32_t last_tok = fast_div(last_row, div_g);
     if (last_tok > (uint32_t)(n - 1)) last_tok = (uint32_t)(n - 1);
     return (int)(((uint32_t)L + last_tok + 1u + (uint32_t)kTileN - 1u) / (uint32_t)kTileN);
+}
+
+// KV tiles of unit u of a SHARED-PREFIX batch item: the first L tokens of a cache that several items
+// share (all of them visible to every row), then the item's own n new tokens from a separate buffer
+// (causal).  The two parts are tiled separately: the own tokens start a new tile.
+__host__ __device__ inline int tail_kv_tiles(int L, int n, int G, int unit, int unit_rows)
+{
+    unsigned last_row = (unsigned)(unit + 1) * (unsigned)unit_rows - 1u;
+    unsigned last_tok = last_row / (unsigned)G;
+    if (last_tok > (unsigned)(n - 1)) last_tok = (unsigned)(n - 1);
+    return (int)(((unsigned)L + (unsigned)kTileN - 1u) / (unsigned)kTileN + (last_tok + (unsigned)kTileN) / (unsigned)kTileN);
+}
+__host__ __device__ inline int tail_kv_tiles_fast(int L, int n, FastDiv div_g, int unit, int unit_rows)
+{
+    const uint32_t last_row = (uint32_t)(unit + 1) * (uint32_t)unit_rows - 1u;
+    uint32_t last_tok = fast_div(last_row, div_g);
+    if (last_tok > (uint32_t)(n - 1)) last_tok = (uint32_t)(n - 1);
+    return (int)(((uint32_t)L + (uint32_t)kTileN - 1u) / (uint32_t)kTileN + (last_tok + (uint32_t)kTileN) / (uint32_t)kTileN);
+}
+
+// Where token m of a dense run of tokens sits in a PACKED sequence I, v_1, a_1, ..., v_N, a_N
+// (Sec. 3.3): `action` = 0 maps the run instruction + visual tokens, 1 the run of action tokens.
+// F = 0 means "not packed": the identity.
+struct PackedMap {
+    int I, F, A, action;
+};
+__host__ __device__ inline long packed_row(const PackedMap& pm, long m)
+{
+    if (pm.F <= 0 && pm.A <= 0) return m;
+    if (pm.action) return pm.I + (m / pm.A) * (long)(pm.F + pm.A) + pm.F + m % pm.A;
+    if (m < pm.I || pm.F <= 0) return m;
+    return pm.I + ((m - pm.I) / pm.F) * (long)(pm.F + pm.A) + (m - pm.I) % pm.F;
 }
 
 // Stub lengths for the kernels that serve one episode.

@@ -8,8 +8,10 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <utility>
+#include <vector>
 
 #include "attn_simt.cuh"
 #include "attn_pair.cuh"
@@ -110,6 +112,22 @@ evlnStatus_t cuda_fail(evlnHandle_t h, cudaError_t e)
     return EVLN_CUDA_ERROR;
 }
 
+// The handle's device must be current when work is launched: the kernels' attributes and the
+// tensor maps belong to that device's context.
+bool device_is_current(evlnHandle_t h)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
+
+// An optional position table must cover the positions [first, first + count) of the call.
+bool rope_table_covers(const void* table, int table_first, int table_count, long first, long count)
+{
+    if (!table) return true;
+    if (!aligned16(table) || table_first < 0 || table_count < 0) return false;
+    return (long)table_first <= first && first + count <= (long)table_first + table_count;
+}
+
 evlnStatus_t check_step_params(evlnHandle_t h, const evlnStepParams* p)
 {
     if (!h || !p) return EVLN_INVALID_VALUE;
@@ -124,6 +142,8 @@ evlnStatus_t check_step_params(evlnHandle_t h, const evlnStepParams* p)
     if (p->head_dim != 64 && p->head_dim != 128) return EVLN_NOT_SUPPORTED;
     if ((long)p->cache_len + p->num_new > (long)p->cache_capacity) return EVLN_CACHE_FULL;
     if ((long)p->num_new * p->num_q_heads / p->num_kv_heads > (1 << 24)) return EVLN_NOT_SUPPORTED;
+    if (!rope_table_covers(p->rope_table, p->rope_table_first_pos, p->rope_table_count, p->cache_len, p->num_new))
+        return EVLN_INVALID_VALUE;
     return EVLN_OK;
 }
 
@@ -235,61 +255,78 @@ evlnStatus_t check_paged_params(evlnHandle_t h, const evlnPagedParams* p, const 
     return EVLN_OK;
 }
 
-// Work-item size (KV tiles) and the largest split count of a paged batch.
-void paged_schedule(evlnHandle_t h, const evlnPagedParams* p, const int* lens, const int* offs,
-                    int* chunk_tiles, int* max_splits, long* items)
+// KV tiles of unit u of a batch item: paged episode, or item sharing a cache prefix (tail).
+inline int batch_kv_tiles(bool tail, int L, int n, int G, int u)
 {
-    const int G = p->num_q_heads / p->num_kv_heads;
+    return tail ? tail_kv_tiles(L, n, G, u, kUnitRows) : unit_kv_tiles(L, n, G, u, kUnitRows);
+}
+
+// Work-item size (KV tiles) and the largest split count of a batch.
+void batch_schedule(int num_sms, int G, int Hkv, int batch, const int* lens, const int* offs, bool tail,
+                    int kv_chunk_tiles, int* chunk_tiles, int* max_splits, long* items)
+{
     long total = 0;
     int nkv_max = 1;
-    for (int b = 0; b < p->batch; ++b) {
+    for (int b = 0; b < batch; ++b) {
         const int n = offs[b + 1] - offs[b];
         const int units = ceil_div(n * G, kUnitRows);
         for (int u = 0; u < units; ++u) {
-            const int nkv = unit_kv_tiles(lens[b], n, G, u, kUnitRows);
+            const int nkv = batch_kv_tiles(tail, lens[b], n, G, u);
             total += nkv;
             if (nkv > nkv_max) nkv_max = nkv;
         }
     }
-    total *= p->num_kv_heads;
-    int chunk = p->kv_chunk_tiles;
+    total *= Hkv;
+    int chunk = kv_chunk_tiles;
     if (chunk <= 0) {
-        const long pairs = h->num_sms / 2 > 0 ? h->num_sms / 2 : 1;
+        const long pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
         chunk = (int)((total + pairs * 4 - 1) / (pairs * 4));
         if (chunk < 8) chunk = 8;
     }
     if (chunk < ceil_div(nkv_max, kMaxSplits)) chunk = ceil_div(nkv_max, kMaxSplits);
     long cnt = 0;
-    for (int b = 0; b < p->batch; ++b) {
+    for (int b = 0; b < batch; ++b) {
         const int n = offs[b + 1] - offs[b];
         const int units = ceil_div(n * G, kUnitRows);
-        for (int u = 0; u < units; ++u) cnt += ceil_div(unit_kv_tiles(lens[b], n, G, u, kUnitRows), chunk);
+        for (int u = 0; u < units; ++u) cnt += ceil_div(batch_kv_tiles(tail, lens[b], n, G, u), chunk);
     }
     *chunk_tiles = chunk;
     *max_splits = ceil_div(nkv_max, chunk);
-    *items = cnt * p->num_kv_heads;
+    *items = cnt * Hkv;
+}
+
+void paged_schedule(evlnHandle_t h, const evlnPagedParams* p, const int* lens, const int* offs,
+                    int* chunk_tiles, int* max_splits, long* items)
+{
+    batch_schedule(h->num_sms, p->num_q_heads / p->num_kv_heads, p->num_kv_heads, p->batch, lens, offs, false,
+                   p->kv_chunk_tiles, chunk_tiles, max_splits, items);
 }
 
 // chunk_tiles > 0: also the first attention work item of every episode (items are numbered
 // episode by episode: kv head, unit, split)
-void fill_lens(BatchLens* bl, const evlnPagedParams* p, const int* lens, const int* offs, int chunk_tiles = 0)
+void fill_batch_lens(BatchLens* bl, int G, int Hkv, int batch, const int* lens, const int* offs, int chunk_tiles, bool tail)
 {
     memset(bl, 0, sizeof(*bl));
-    for (int b = 0; b < p->batch; ++b) bl->cache_len[b] = lens[b];
-    for (int b = 0; b <= p->batch; ++b) bl->new_off[b] = offs[b];
+    for (int b = 0; b < batch; ++b) bl->cache_len[b] = lens[b];
+    for (int b = 0; b <= batch; ++b) bl->new_off[b] = offs[b];
+    for (int b = batch + 1; b <= kMaxBatch; ++b) bl->new_off[b] = offs[batch];
     if (chunk_tiles > 0) {
-        const int G = p->num_q_heads / p->num_kv_heads;
         int items = 0;
-        for (int b = 0; b < p->batch; ++b) {
+        for (int b = 0; b < batch; ++b) {
             bl->item_off[b] = items;
             const int n = offs[b + 1] - offs[b];
             const int units = ceil_div(n * G, kUnitRows);
             int per_head = 0;
-            for (int u = 0; u < units; ++u) per_head += ceil_div(unit_kv_tiles(lens[b], n, G, u, kUnitRows), chunk_tiles);
-            items += per_head * p->num_kv_heads;
+            for (int u = 0; u < units; ++u) per_head += ceil_div(batch_kv_tiles(tail, lens[b], n, G, u), chunk_tiles);
+            items += per_head * Hkv;
         }
-        for (int b = p->batch; b <= kMaxBatch; ++b) bl->item_off[b] = items;
+        for (int b = batch; b <= kMaxBatch; ++b) bl->item_off[b] = items;
     }
+}
+
+void fill_lens(BatchLens* bl, const evlnPagedParams* p, const int* lens, const int* offs, int chunk_tiles = 0)
+{
+    fill_batch_lens(bl, p->num_q_heads / p->num_kv_heads, p->num_kv_heads, p->batch, lens, offs, chunk_tiles, false);
 }
 
 template <typename T>
@@ -308,6 +345,8 @@ evlnStatus_t launch_combine(evlnHandle_t h, const CombineArgs& a, int D, bool pa
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
+
+evlnStatus_t noalloc_status_word(int** word);     // defined with the allocation-free variant below
 
 }  // namespace
 
@@ -337,7 +376,14 @@ evlnStatus_t evlnCreate(evlnHandle_t* handle, int device)
     h->last_cuda_error = 0;
     h->d_status = nullptr;
     h->encode = nullptr;
-    cudaError_t e = cudaSetDevice(device);
+    int prev_device = -1;
+    cudaError_t e = cudaGetDevice(&prev_device);
+    if (e == cudaSuccess) e = cudaSetDevice(device);
+    // whatever happens below, the caller's current device is put back
+    struct Restore {
+        int dev;
+        ~Restore() { if (dev >= 0) cudaSetDevice(dev); }
+    } restore{prev_device};
     cudaDeviceProp prop;
     if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, device);
     if (e != cudaSuccess) { delete h; return EVLN_CUDA_ERROR; }
@@ -384,15 +430,70 @@ int evlnGetLastCudaError(evlnHandle_t h) { return h ? h->last_cuda_error : 0; }
 
 evlnStatus_t evlnGetDeviceStatus(evlnHandle_t h, void* stream, int* device_status)
 {
-    if (!h || !device_status) return EVLN_INVALID_VALUE;
+    if (!device_status) return EVLN_INVALID_VALUE;
+    int* word = nullptr;
+    if (h) {
+        if (!device_is_current(h)) return EVLN_INVALID_VALUE;
+        word = h->d_status;
+    } else {
+        // the allocation-free call's status word on the current device (part of the library image)
+        evlnStatus_t s = noalloc_status_word(&word);
+        if (s != EVLN_OK) return s;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     int v = 0;
-    cudaError_t e = cudaMemcpyAsync(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, st);
+    cudaError_t e = cudaMemcpyAsync(&v, word, sizeof(int), cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    if (e == cudaSuccess && v != 0) e = cudaMemsetAsync(h->d_status, 0, sizeof(int), st);
-    if (e != cudaSuccess) return cuda_fail(h, e);
+    if (e == cudaSuccess && v != 0) e = cudaMemsetAsync(word, 0, sizeof(int), st);
+    if (e != cudaSuccess) return h ? cuda_fail(h, e) : EVLN_CUDA_ERROR;
     *device_status = v;
     return v == 0 ? EVLN_OK : EVLN_DEVICE_TIMEOUT;
+}
+
+// A bounded wait on a barrier nobody arrives on: it must run out and leave its code in the status word.
+__global__ void selftest_wait_kernel(int* status, long long limit_cycles)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int s_abort;
+    const uint32_t b = ptx::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        ptx::mbar_init(b, 1);
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) wait_bounded(b, 0, EVLN_SELFTEST_STATUS_CODE, status, &s_abort, limit_cycles);
+    __syncthreads();
+}
+
+evlnStatus_t evlnSelfTestBoundedWait(evlnHandle_t h, long long limit_cycles, void* stream)
+{
+    if (!h || limit_cycles < 1000 || limit_cycles > 1000000000LL) return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
+    selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(h->d_status, limit_cycles);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+size_t evlnRopeTableBytes(int head_dim, int count)
+{
+    if ((head_dim != 64 && head_dim != 128) || count < 0) return 0;
+    return (size_t)count * (head_dim / 2) * sizeof(double2);
+}
+
+evlnStatus_t evlnRopeTable(evlnHandle_t h, int head_dim, double rope_theta, int first_pos, int count, void* table,
+                           void* stream)
+{
+    if (!h || first_pos < 0 || count < 0 || !(rope_theta > 0.0)) return EVLN_INVALID_VALUE;
+    if (head_dim != 64 && head_dim != 128) return EVLN_NOT_SUPPORTED;
+    if (count == 0) return EVLN_OK;
+    if (!table || !aligned16(table)) return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
+    const long total = (long)count * (head_dim / 2);
+    launch_pdl(rope_table_kernel, dim3((unsigned)((total + 127) / 128)), dim3(128), 0, (cudaStream_t)stream,
+               (double2*)table, first_pos, count, head_dim, log2(rope_theta));
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
 
 evlnStatus_t evlnStepNumSplits(evlnHandle_t h, const evlnStepParams* p, int* num_splits)
@@ -434,6 +535,7 @@ evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void*
     if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(q_rot) ||
         !aligned16(k_cache) || !aligned16(v_cache))
         return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     const int vec = 16 / elem_bytes(p->dtype);
     if (q_stride_tok < (long)p->num_q_heads * p->head_dim || k_stride_tok < (long)p->num_kv_heads * p->head_dim ||
         v_stride_tok < (long)p->num_kv_heads * p->head_dim)
@@ -448,6 +550,8 @@ evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void*
     a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
     a.cache_len = p->cache_len; a.num_new = p->num_new; a.cache_cap = p->cache_capacity;
     a.log2_theta = log2(p->rope_theta);
+    a.table = (const double2*)p->rope_table;
+    a.table_first = p->rope_table_first_pos;
     NoLens nl = {};
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16)
@@ -467,6 +571,7 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
     if (!q_rot || !k_cache || !v_cache || !workspace) return EVLN_INVALID_VALUE;
     if (!aligned16(q_rot) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(workspace))
         return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     const int G = p->num_q_heads / p->num_kv_heads;
     const int R = p->num_new * G;
     const int D = p->head_dim;
@@ -542,6 +647,7 @@ evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void
     if (s != EVLN_OK) return s;
     if (p->num_new == 0) return EVLN_OK;
     if (!workspace || !out || !aligned16(workspace) || !aligned16(out)) return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     const int G = p->num_q_heads / p->num_kv_heads;
     const int R = p->num_new * G;
     const int S = resolve_splits(h, p);
@@ -604,6 +710,7 @@ evlnStatus_t evlnPagedRopeAppend(evlnHandle_t h, const evlnPagedParams* p, const
     if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(q_rot) ||
         !aligned16(k_pool) || !aligned16(v_pool))
         return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     RopeArgs a = {};
     a.q_new = q_new; a.k_new = k_new; a.v_new = v_new;
     a.q_rot = q_rot; a.k_cache = k_pool; a.v_cache = v_pool; a.page_table = d_page_table;
@@ -631,6 +738,7 @@ evlnStatus_t evlnPagedStepAttention(evlnHandle_t h, const evlnPagedParams* p, co
     if (!q_rot || !k_pool || !v_pool || !d_page_table || !workspace) return EVLN_INVALID_VALUE;
     if (!aligned16(q_rot) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(workspace))
         return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     const int G = p->num_q_heads / p->num_kv_heads;
     const long rows = (long)total * G;
     int chunk, smax;
@@ -681,6 +789,7 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t h, const evlnPagedParams* p, cons
     const int total = h_new_offsets[p->batch];
     if (total == 0) return EVLN_OK;
     if (!workspace || !out || !aligned16(workspace) || !aligned16(out)) return EVLN_INVALID_VALUE;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     const int G = p->num_q_heads / p->num_kv_heads;
     const long rows = (long)total * G;
     int chunk, smax;
@@ -697,6 +806,32 @@ evlnStatus_t evlnPagedStepCombine(evlnHandle_t h, const evlnPagedParams* p, cons
     return launch_combine<__nv_bfloat16>(h, a, 128, true, &bl, (cudaStream_t)stream);
 }
 
+evlnStatus_t evlnPagedCheckTable(const evlnPagedParams* p, const int* h_cache_lens, const int* h_new_offsets,
+                                 const int* h_page_table, int* h_bad_episode, int* h_bad_index)
+{
+    if (!p || !h_cache_lens || !h_new_offsets || !h_page_table) return EVLN_INVALID_VALUE;
+    if (p->struct_size != sizeof(evlnPagedParams)) return EVLN_INVALID_VALUE;
+    if (p->batch < 1 || p->num_pages < 1 || p->max_pages_per_seq < 1 || p->page_size < 1) return EVLN_INVALID_VALUE;
+    if (h_new_offsets[0] != 0) return EVLN_INVALID_VALUE;
+    std::vector<unsigned char> used((size_t)p->num_pages, 0);
+    for (int b = 0; b < p->batch; ++b) {
+        if (h_cache_lens[b] < 0 || h_new_offsets[b + 1] < h_new_offsets[b]) return EVLN_INVALID_VALUE;
+        const long tokens = (long)h_cache_lens[b] + (h_new_offsets[b + 1] - h_new_offsets[b]);
+        const long need = (tokens + p->page_size - 1) / p->page_size;
+        if (need > p->max_pages_per_seq) return EVLN_CACHE_FULL;
+        for (long i = 0; i < need; ++i) {
+            const int pg = h_page_table[(long)b * p->max_pages_per_seq + i];
+            if (pg < 0 || pg >= p->num_pages || used[pg]) {
+                if (h_bad_episode) *h_bad_episode = b;
+                if (h_bad_index) *h_bad_index = (int)i;
+                return EVLN_INVALID_VALUE;
+            }
+            used[pg] = 1;
+        }
+    }
+    return EVLN_OK;
+}
+
 }  // extern "C"
 
 // ---- un-rotated store + frame sampler ------------------------------------------------------
@@ -710,6 +845,7 @@ evlnStatus_t check_gather_params(evlnHandle_t h, const evlnGatherParams* p)
     if (p->num_kv_heads <= 0 || p->store_capacity < 0 || p->work_capacity < 0) return EVLN_INVALID_VALUE;
     if (!(p->rope_theta > 0.0)) return EVLN_INVALID_VALUE;
     if (p->head_dim != 64 && p->head_dim != 128) return EVLN_NOT_SUPPORTED;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
     return EVLN_OK;
 }
 }  // namespace
@@ -786,6 +922,7 @@ extern "C" evlnStatus_t evlnGatherRope(evlnHandle_t h, const evlnGatherParams* p
     for (int i = num_segments; i <= kMaxSegments; ++i) segs.dst_off[i] = (int)total;
     if (h_total) *h_total = (int)total;
     if (total == 0) return EVLN_OK;
+    if (!rope_table_covers(p->rope_table, p->rope_table_first_pos, p->rope_table_count, 0, total)) return EVLN_INVALID_VALUE;
     if (!k_store || !v_store || !k_work || !v_work) return EVLN_INVALID_VALUE;
     if (!aligned16(k_store) || !aligned16(v_store) || !aligned16(k_work) || !aligned16(v_work)) return EVLN_INVALID_VALUE;
     GatherArgs a = {};
@@ -794,6 +931,8 @@ extern "C" evlnStatus_t evlnGatherRope(evlnHandle_t h, const evlnGatherParams* p
     a.src_cap = p->store_capacity; a.dst_cap = p->work_capacity;
     a.num_tokens = (int)total; a.num_segments = num_segments;
     a.log2_theta = log2(p->rope_theta);
+    a.table = (const double2*)p->rope_table;
+    a.table_first = p->rope_table_first_pos;
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16) launch_pdl(gather_rope_kernel<__nv_bfloat16>, dim3((int)total), dim3(128), 0, st, a, segs);
     else launch_pdl(gather_rope_kernel<float>, dim3((int)total), dim3(128), 0, st, a, segs);
@@ -851,7 +990,7 @@ extern "C" evlnStatus_t evlnStoreFetch(evlnHandle_t h, const evlnGatherParams* p
 // names below are only stand-ins for the device objects; their device addresses come from
 // cudaGetSymbolAddress (once per device) and are what the kernels receive.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[EVLN_NOALLOC_SCRATCH_BYTES];
-static __device__ __align__(256) int g_noalloc_status[64];
+static __device__ __align__(256) int g_noalloc_status;
 
 namespace {
 constexpr int kMaxDevices = 64;
@@ -861,12 +1000,14 @@ struct NoAllocDevice {
     void* scratch;
 };
 NoAllocDevice g_noalloc_dev[kMaxDevices];
+std::mutex g_noalloc_mutex;       // host threads may race for the first call on a device
 
 // First call on a device: resolve device addresses and properties.  Allocates nothing.
 evlnStatus_t noalloc_setup(int device, NoAllocDevice** out)
 {
     if (device < 0 || device >= kMaxDevices) return EVLN_NOT_SUPPORTED;
     NoAllocDevice* d = &g_noalloc_dev[device];
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     if (!d->ready) {
         cudaDeviceProp prop;
         cudaError_t e = cudaGetDeviceProperties(&prop, device);
@@ -897,6 +1038,17 @@ evlnStatus_t noalloc_setup(int device, NoAllocDevice** out)
         d->ready = true;
     }
     *out = d;
+    return EVLN_OK;
+}
+// Device address of the allocation-free call's status word on the current device.
+evlnStatus_t noalloc_status_word(int** word)
+{
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return EVLN_CUDA_ERROR;
+    NoAllocDevice* d = nullptr;
+    evlnStatus_t s = noalloc_setup(device, &d);
+    if (s != EVLN_OK) return s;
+    *word = d->ctx.d_status;
     return EVLN_OK;
 }
 }  // namespace

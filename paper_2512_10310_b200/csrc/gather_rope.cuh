@@ -5,11 +5,13 @@
 // store_append_kernel: the new frame's raw (un-rotated) K and V go to the store, head-major.
 // gather_rope_kernel: the kept segments of the store are laid out back to back in a working cache;
 // the token that lands in working slot p is rotated at position p (keys) or copied (values).  One
-// CTA per destination token; angles in double precision as in the append kernel.  HBM-bound: every
+// CTA per destination token; angles in double precision as in the append kernel (or from the
+// caller's position table).  HBM-bound: every
 // kept element is read once and written once with 128-bit accesses.
 #pragma once
 
 #include "common.cuh"
+#include "rope_append.cuh"
 
 namespace evln {
 
@@ -34,6 +36,8 @@ struct GatherArgs {
     int num_tokens;         // destination tokens
     int num_segments;       // gather only
     double log2_theta;      // gather only
+    const double2* table;   // gather only, optional: (cos, sin) per (position - table_first, j)
+    int table_first;
 };
 
 template <typename T>
@@ -77,11 +81,9 @@ gather_rope_kernel(const GatherArgs a, const __grid_constant__ SegList segs)
 
     if (threadIdx.x < half) {
         const int j = threadIdx.x;
-        const double omega = exp2(-(2.0 * (double)j / (double)D) * a.log2_theta);
-        double s, c;
-        sincospi((double)pos * omega * 0.31830988618379067154, &s, &c);
-        s_cos[j] = c;
-        s_sin[j] = s;
+        const double2 cs = a.table ? a.table[(long)(pos - a.table_first) * half + j] : rope_cos_sin(pos, j, D, a.log2_theta);
+        s_cos[j] = cs.x;
+        s_sin[j] = cs.y;
     }
     __syncthreads();
 

@@ -66,25 +66,10 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
-                                            int x, int y, int z, int w)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
-        : "memory");
-}
 // L2 prefetch of a tile (no shared-memory destination, no barrier)
 __device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int x, int y, int z)
 {
     asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int x, int y, int z, int w)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(x), "r"(y), "r"(z),
-                 "r"(w)
                  : "memory");
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map)
@@ -229,10 +214,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void cluster_arrive()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-}
 // arrival without the cluster-wide release of this thread's earlier writes (a flush that costs about
 // a thousand cycles): for meetings whose only shared state is ordered by fences of its own
 // (fence.mbarrier_init for the barriers, tcgen05 fences for tensor memory)
@@ -357,6 +338,8 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// Registers per thread of the executing warpgroup (all four warps execute it together): dec gives
+// registers back to the CTA's pool, inc takes from it and WAITS until the pool can serve it.
 template <int N> __device__ __forceinline__ void setmaxnreg_inc()
 {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));

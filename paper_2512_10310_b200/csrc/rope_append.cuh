@@ -1,11 +1,14 @@
 // Fused RoPE-rotate-and-append kernel (Sec. 3.2: contiguous position ids, rotation,
 // concatenation of the new frame with the reused cache).
 //
-// One CTA per new token.  Phase 1: D/2 threads form the token's angles phi_j = pos * theta^(-2j/D)
+// One CTA per new token.  Phase 1: D/2 threads get the token's cos/sin of phi_j = pos * theta^(-2j/D)
 // in double precision (pos reaches tens of thousands; a float angle would be off by ~1e-3 rad)
-// and leave cos/sin (double) in shared memory for all heads.  Phase 2: every thread moves 16-byte
+// into shared memory for all heads: from the caller's position table when there is one (the
+// table depends on the positions only, so a model makes it once per navigation step for all its
+// layers: rope_table_kernel below), else formed on the spot.  Phase 2: every thread moves 16-byte
 // vectors: rotated query halves to the kv-head-grouped q_rot scratch, rotated key halves and
-// the unchanged values to the token's cache slot.  HBM-bound: each element is read once and
+// the unchanged values to the token's cache slot; the loads of a thread's first vectors are
+// issued before the trigonometry is waited for.  HBM-bound: each element is read once and
 // written once with 128-bit accesses.
 #pragma once
 
@@ -28,7 +31,36 @@ struct RopeArgs {
     int cache_cap;      // contiguous only
     int batch, page_size, max_pages;     // paged only
     double log2_theta;
+    const double2* table;   // optional: (cos, sin) per (position - table_first, j), [count][D/2]
+    int table_first;
+    int tail;               // batch mode without pages: K/V of new token m go to row m of k_cache / v_cache
+                            // = buffers [Hkv, total new tokens, D] (the items' own tokens, not a shared cache)
+    PackedMap map;          // where new token m sits in q_new / k_new / v_new (identity unless packed)
 };
+
+// cos/sin of pos * theta^(-2j/D): the one definition the append, gather and table kernels share
+__device__ __forceinline__ double2 rope_cos_sin(long pos, int j, int D, double log2_theta)
+{
+    const double omega = exp2(-(2.0 * (double)j / (double)D) * log2_theta);
+    double s, c;
+    // sin/cos(pos * omega) through sincospi: its range reduction is exact and cheap, where a
+    // plain sincos of an argument of thousands of radians takes the slow reduction path
+    sincospi((double)pos * omega * 0.31830988618379067154, &s, &c);
+    return make_double2(c, s);
+}
+
+// Position table: entry (p, j) = (cos, sin) of (first_pos + p) * theta^(-2j/D).
+__global__ void __launch_bounds__(128)
+rope_table_kernel(double2* table, int first_pos, int count, int D, double log2_theta)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int half = D / 2;
+    const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long)count * half) return;
+    const int p = (int)(i / half), j = (int)(i % half);
+    table[i] = rope_cos_sin((long)first_pos + p, j, D, log2_theta);
+}
 
 // LensT is BatchLens for the paged kernel and NoLens (a stub) for the contiguous one.
 
@@ -62,32 +94,29 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
 
     if (threadIdx.x < half) {
         const int j = threadIdx.x;
-        double omega = exp2(-(2.0 * (double)j / (double)D) * a.log2_theta);
-        double s, c;
-        // sin/cos(pos * omega) through sincospi: its range reduction is exact and cheap, where a
-        // plain sincos of an argument of thousands of radians takes the slow reduction path
-        sincospi((double)pos * omega * 0.31830988618379067154, &s, &c);
-        s_cos[j] = c;
-        s_sin[j] = s;
+        const double2 cs = a.table ? a.table[(pos - a.table_first) * half + j] : rope_cos_sin(pos, j, D, a.log2_theta);
+        s_cos[j] = cs.x;
+        s_sin[j] = cs.y;
     }
-    __syncthreads();
 
     // destination of this token's K/V row for kv head g (element offset)
     long page_base = 0;     // paged: (page_id * Hkv) * page_size * D, slot within page
     int slot = 0;
-    if (PAGED) {
+    if (PAGED && !a.tail) {
         int pg = a.page_table[(long)b * a.max_pages + (int)(pos / a.page_size)];
         slot = (int)(pos % a.page_size);
         page_base = (long)pg * a.Hkv * a.page_size * D;
     }
     auto kv_row = [&](int g) -> long {
+        if (PAGED && a.tail) return ((long)g * lens.new_off[a.batch] + tok) * D;
         if (PAGED) return page_base + ((long)g * a.page_size + slot) * D;
         return ((long)g * a.cache_cap + pos) * D;
     };
 
-    const T* q_tok = (const T*)a.q_new + (long)tok * a.q_stride;
-    const T* k_tok = (const T*)a.k_new + (long)tok * a.k_stride;
-    const T* v_tok = (const T*)a.v_new + (long)tok * a.v_stride;
+    const long src_tok = packed_row(a.map, tok);
+    const T* q_tok = (const T*)a.q_new + src_tok * a.q_stride;
+    const T* k_tok = (const T*)a.k_new + src_tok * a.k_stride;
+    const T* v_tok = (const T*)a.v_new + src_tok * a.v_stride;
 
     const int vec_per_half = half / V;
     const int q_items = a.Hq * vec_per_half;
@@ -96,13 +125,30 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
     const int items = q_items + k_items + v_items;
     const long rows_per_head = PAGED ? (long)lens.new_off[a.batch] * G : (long)a.num_new * G;
 
-    for (int it = threadIdx.x; it < items; it += blockDim.x) {
+    // a thread's work item `it`: a pair of 16-byte vectors (j0.., j0+half..) of a query or key head,
+    // or one 16-byte vector of a value head
+    auto load_item = [&](int it, uint4& r0, uint4& r1) {
         if (it < q_items + k_items) {
             const bool is_q = it < q_items;
             const int e = is_q ? it : it - q_items;
             const int h = e / vec_per_half;
             const int j0 = (e % vec_per_half) * V;
             const T* src = (is_q ? q_tok : k_tok) + (long)h * D;
+            r0 = *reinterpret_cast<const uint4*>(src + j0);
+            r1 = *reinterpret_cast<const uint4*>(src + j0 + half);
+        } else {
+            const int e = it - q_items - k_items;
+            const int g = e / (D / V);
+            const int d0 = (e % (D / V)) * V;
+            r0 = *reinterpret_cast<const uint4*>(v_tok + (long)g * D + d0);
+        }
+    };
+    auto finish_item = [&](int it, const uint4& lo_raw, const uint4& hi_raw) {
+        if (it < q_items + k_items) {
+            const bool is_q = it < q_items;
+            const int e = is_q ? it : it - q_items;
+            const int h = e / vec_per_half;
+            const int j0 = (e % vec_per_half) * V;
             T* dst;
             if (is_q) {
                 const int g = h / G;
@@ -110,8 +156,6 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
             } else {
                 dst = (T*)a.k_cache + kv_row(h);
             }
-            uint4 lo_raw = *reinterpret_cast<const uint4*>(src + j0);
-            uint4 hi_raw = *reinterpret_cast<const uint4*>(src + j0 + half);
             const T* lo = reinterpret_cast<const T*>(&lo_raw);
             const T* hi = reinterpret_cast<const T*>(&hi_raw);
             uint4 out_lo_raw, out_hi_raw;
@@ -132,12 +176,20 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
             const int e = it - q_items - k_items;
             const int g = e / (D / V);
             const int d0 = (e % (D / V)) * V;
-            uint4 raw = *reinterpret_cast<const uint4*>(v_tok + (long)g * D + d0);
-            *reinterpret_cast<uint4*>((T*)a.v_cache + kv_row(g) + d0) = raw;
+            *reinterpret_cast<uint4*>((T*)a.v_cache + kv_row(g) + d0) = lo_raw;
         }
+    };
+
+    uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
+    if ((int)threadIdx.x < items) load_item(threadIdx.x, r0, r1);     // in flight while the cos/sin arrive
+    __syncthreads();
+    if ((int)threadIdx.x < items) finish_item(threadIdx.x, r0, r1);
+    for (int it = threadIdx.x + blockDim.x; it < items; it += blockDim.x) {
+        load_item(it, r0, r1);
+        finish_item(it, r0, r1);
     }
 
-    if (PAGED && i == n_b - 1 && slot + 1 < a.page_size) {
+    if (PAGED && !a.tail && i == n_b - 1 && slot + 1 < a.page_size) {
         // the episode's last page is only partly filled: clear the value slots behind the last
         // token so that a tile load of the whole page never brings in stale bits
         const int tail = a.page_size - (slot + 1);

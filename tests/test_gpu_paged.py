@@ -64,9 +64,10 @@ def _check_pools(x, cfg, k_pool, v_pool, ok_pool, ov_pool):
             pg, sl = x["page_table"][b][t // P], t % P
             assert bf16_ulp_distance(k_pool[pg, :, sl], ok_pool[pg, sl]).max() <= 1
             assert np.array_equal(f64(v_pool[pg, :, sl]), ov_pool[pg, sl])
-        # value slots behind the last token of the last page are cleared
+        # value slots behind the last appended token of the last page are cleared (an episode that
+        # appends nothing this step is not touched, and nothing of it is read)
         last = L + n
-        if last % P:
+        if n > 0 and last % P:
             pg = x["page_table"][b][last // P]
             assert bool((v_pool[pg, :, last % P:] == 0).all())
 
@@ -101,33 +102,52 @@ def test_paged_equals_contiguous_on_device(handle):
     assert (g["lse"] - lse).abs().max().item() <= 1e-5
 
 
-def test_paged_b16_full_size_sampled(handle):
-    # the full serving batch; the oracle checks sampled tokens of sampled episodes one by one
+def test_paged_b16_full_size_all_rows(handle):
+    # the full serving batch (16 episodes, L from 1024 to 16384, 196 new tokens each): every output row,
+    # every log-sum-exp and every appended slot against the oracle
     cfg = W.PAGED_B16
     x = W.make_paged_inputs(cfg)
     out, lse, k_pool, v_pool = _gpu_paged(handle, cfg, x)
-    P, theta = cfg.page_size, cfg.rope_theta
-    lens, offs = x["cache_lens"], x["new_offsets"]
-    order = np.argsort(lens)
-    for b in (int(order[0]), int(order[len(order) // 2]), int(order[-1])):
-        L, lo, hi = lens[b], offs[b], offs[b + 1]
-        n = hi - lo
-        pages = x["page_table"][b]
-        kc = np.zeros((L + n, cfg.num_kv_heads, cfg.head_dim))
-        vc = np.zeros_like(kc)
-        kc[:L] = f64(torch.cat([x["k_pool"][pg] for pg in pages])[:L])
-        vc[:L] = f64(torch.cat([x["v_pool"][pg] for pg in pages])[:L])
-        kc[L:] = so.round_bf16(so.rope(f64(x["k_new"][lo:hi]), L, theta))
-        vc[L:] = f64(x["v_new"][lo:hi])
-        q_rot = so.rope(f64(x["q_new"][lo:hi]), L, theta)
-        for i in (0, 18, 100, n - 1):
-            o, l = so.attend_range(q_rot[i:i + 1], kc, vc, L + i, 0, L + i + 1)
-            check_output("bf16", out[lo + i:lo + i + 1], lse[lo + i:lo + i + 1], o, l)
-        # appended slots of this episode
-        for t in (L, L + n - 1):
-            pg, sl = pages[t // P], t % P
-            assert bf16_ulp_distance(k_pool[pg, :, sl], kc[t]).max() <= 1
-            assert np.array_equal(f64(v_pool[pg, :, sl]), vc[t])
+    okp, ovp = f64(x["k_pool"]), f64(x["v_pool"])
+    ref_out, ref_lse = so.step_paged(f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"]), okp, ovp,
+                                     x["page_table"], x["cache_lens"], x["new_offsets"], cfg.rope_theta, storage="bf16")
+    check_output("bf16", out, lse, ref_out, ref_lse)
+    _check_pools(x, cfg, k_pool, v_pool, okp, ovp)
+    # ... and episode by episode, so that a short episode cannot hide behind the long ones' norm
+    for b in range(cfg.batch):
+        lo, hi = x["new_offsets"][b], x["new_offsets"][b + 1]
+        check_output("bf16", out[lo:hi], lse[lo:hi], ref_out[lo:hi], ref_lse[lo:hi])
+
+
+def test_paged_episodes_without_new_tokens(handle):
+    # episodes that contribute no token this step: first, in the middle and last of the batch
+    cfg = dataclasses.replace(W.PAGED_B16, name="paged_idle", batch=6, seed=33)
+    lens = [500, 130, 64, 900, 257, 300]
+    news = [0, 70, 0, 196, 129, 0]
+    x = W.make_paged_inputs(cfg, lens=lens, num_new=news)
+    for chunk in (0, 3):
+        out, lse, k_pool, v_pool = _gpu_paged(handle, cfg, x, kv_chunk_tiles=chunk)
+        okp, ovp = f64(x["k_pool"]), f64(x["v_pool"])
+        ref_out, ref_lse = so.step_paged(f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"]), okp, ovp,
+                                         x["page_table"], lens, x["new_offsets"], cfg.rope_theta, storage="bf16")
+        check_output("bf16", out, lse, ref_out, ref_lse)
+        _check_pools(x, cfg, k_pool, v_pool, okp, ovp)
+
+
+def test_page_table_check_accepts_the_workload_and_names_a_bad_entry(handle):
+    cfg = dataclasses.replace(W.PAGED_B16, name="paged_check", batch=3, seed=34)
+    x = W.make_paged_inputs(cfg, lens=[100, 700, 64], num_new=[30, 196, 1])
+    max_pages = max(len(t) for t in x["page_table"]) + 2
+    p = B.paged_params(cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, 3, cfg.page_size, x["num_pages"], max_pages,
+                       cfg.rope_theta)
+    rows = [t + [0] * (max_pages - len(t)) for t in x["page_table"]]      # padding entries are not looked at
+    assert B.evlnPagedCheckTable(p, x["cache_lens"], x["new_offsets"], rows) == (B.EVLN_OK, -1, -1)
+    bad = [list(r) for r in rows]
+    bad[1][3] = bad[0][1]                      # a page of episode 0 handed to episode 1 as well
+    assert B.evlnPagedCheckTable(p, x["cache_lens"], x["new_offsets"], bad) == (B.EVLN_INVALID_VALUE, 1, 3)
+    bad = [list(r) for r in rows]
+    bad[2][0] = x["num_pages"]                 # outside the pool
+    assert B.evlnPagedCheckTable(p, x["cache_lens"], x["new_offsets"], bad) == (B.EVLN_INVALID_VALUE, 2, 0)
 
 
 def test_paged_argument_errors(handle):

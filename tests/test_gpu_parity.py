@@ -27,7 +27,7 @@ def handle():
 
 
 def _run(handle, cfg, kernel=B.EVLN_KERNEL_AUTO, num_splits=0, extra_cap=37, lse_tol=1e-3, rel_tol=1e-2,
-         inputs=None, round_q=False, abs_tol=1e-2, fused=False):
+         inputs=None, round_q=False, abs_tol=1e-2, fused=False, elem_tol=1e-2):
     x = inputs or W.make_step_inputs(cfg)
     L, n = cfg.cache_len, cfg.num_new
     gs = GpuStep(handle, cfg.dtype, cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n + extra_cap,
@@ -43,7 +43,7 @@ def _run(handle, cfg, kernel=B.EVLN_KERNEL_AUTO, num_splits=0, extra_cap=37, lse
         # rounded q so that the comparison isolates the kernel from that input rounding
         ref_out, ref_lse = so.attend_range(so.round_bf16(r["q_rot"]), r["k_cache"], r["v_cache"], L, 0, L + n)
     check_output(cfg.dtype, g["out"], g["lse"], ref_out, ref_lse, lse_tol=lse_tol, rel_tol=rel_tol,
-                 abs_tol=abs_tol)
+                 abs_tol=abs_tol, elem_tol=elem_tol)
     # rotated queries: bf16 rounding of the oracle's q_rot, at most one ulp apart
     if cfg.dtype == "bf16":
         from tests.helpers import bf16_ulp_distance
@@ -96,7 +96,8 @@ def test_tc_kernel_more_splits_than_tiles(handle):
 def test_tc_kernel_sharp_logits(handle):
     # unit-variance q and k: logits ~ N(0,1), softmax far from uniform
     cfg = dataclasses.replace(W.STEP_7B, name="sharp", cache_len=1500, num_new=100, input_scale=1.0, seed=6)
-    _run(handle, cfg, lse_tol=2e-2, rel_tol=1.5e-2)
+    # (the oracle's unrounded query and the bf16 operand differ by ~1 % in these logits: Frobenius gate only)
+    _run(handle, cfg, lse_tol=2e-2, rel_tol=1.5e-2, elem_tol=None)
 
 
 def test_tc_kernel_planted_high_logit_keys(handle):
@@ -108,8 +109,8 @@ def test_tc_kernel_planted_high_logit_keys(handle):
     x["k_new"][40:42] *= 8.0
     # logits reach ~30 here, so the bf16 rounding of the rotated query alone moves them by ~1e-2;
     # outputs are O(1): the absolute gate scales with them
-    _run(handle, cfg, num_splits=1, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2)
-    _run(handle, cfg, num_splits=3, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2)
+    _run(handle, cfg, num_splits=1, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2, elem_tol=2e-2)
+    _run(handle, cfg, num_splits=3, lse_tol=1e-3, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=4e-2, elem_tol=2e-2)
 
 
 def test_tc_kernel_reference_moves_in_late_tiles(handle):
@@ -126,7 +127,7 @@ def test_tc_kernel_reference_moves_in_late_tiles(handle):
     # the winning scores are several hundred: fp32 accumulation on the tensor core resolves them to
     # a few 1e-5 relative, which is what the log-sum-exp gate allows here
     for splits in (1, 2):
-        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
+        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2, elem_tol=2e-2)
 
 
 # ---- few new tokens: one CTA per (kv head, split) --------------------------------------------
@@ -167,9 +168,9 @@ def test_few_new_tokens_reference_moves(handle):
     x["k_new"][5] *= 250.0
     x["k_new"][7] *= 400.0
     for splits in (1, 2):
-        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2)
+        _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2, elem_tol=2e-2)
         _run(handle, cfg, num_splits=splits, lse_tol=5e-2, rel_tol=1e-2, inputs=x, round_q=True, abs_tol=5e-2,
-             fused=True)
+             fused=True, elem_tol=2e-2)
 
 
 @pytest.mark.parametrize("L,n", [(4096, 196), (4096, 8), (700, 130), (2000, 1), (4090, 8), (20656, 8)])
@@ -292,26 +293,17 @@ def test_chained_steps_reuse_the_cache(handle):
     assert np.array_equal(f64(gs.v_cache[:, :T].permute(1, 0, 2)), vc[:T])
 
 
-def test_long_70b_sampled_rows(handle):
-    # full-size launch; the oracle computes a sample of query tokens one by one
+def test_long_70b_all_rows(handle):
+    # full-size launch (L = 32768, 64 query heads, n = 256); the oracle computes every row
     cfg = W.LONG_70B
     x = W.make_step_inputs(cfg)
     L, n = cfg.cache_len, cfg.num_new
     gs = GpuStep(handle, "bf16", cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, L + n, cfg.rope_theta, n)
     gs.load_cache(x["k_cache"], x["v_cache"])
     g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
-    kc = np.zeros((L + n, cfg.num_kv_heads, cfg.head_dim))
-    vc = np.zeros_like(kc)
-    kc[:L], vc[:L] = f64(x["k_cache"]), f64(x["v_cache"])
-    kc[L:] = so.round_bf16(so.rope(f64(x["k_new"]), L, cfg.rope_theta))
-    vc[L:] = f64(x["v_new"])
-    q_rot = so.rope(f64(x["q_new"]), L, cfg.rope_theta)
-    from tests.helpers import bf16_ulp_distance
-    assert bf16_ulp_distance(gs.k_cache[:, L:].permute(1, 0, 2), kc[L:]).max() <= 1
-    assert np.array_equal(f64(gs.v_cache[:, L:].permute(1, 0, 2)), vc[L:])
-    for i in (0, 1, 127, 128, 200, 255):
-        o, l = so.attend_range(q_rot[i:i + 1], kc, vc, L + i, 0, L + i + 1)
-        check_output("bf16", g["out"][i:i + 1], g["lse"][i:i + 1], o, l)
+    ref = oracle_step("bf16", x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L, cfg.rope_theta)
+    check_cache(gs, ref, L, n)
+    check_output("bf16", g["out"], g["lse"], ref["out"], ref["lse"])
 
 
 # ---- boundary behaviour (argument errors launch nothing) ------------------------------------

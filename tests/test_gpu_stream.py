@@ -1,5 +1,5 @@
 """Streaming episode (instruction prefill + 100 frame steps on a growing cache): the GPU chain
-against the oracle at sampled steps, and the whole appended cache at the end."""
+against the oracle, all rows at the sampled steps, and the whole appended cache at the end."""
 import numpy as np
 import pytest
 import torch
@@ -12,7 +12,7 @@ from tests.helpers import GpuStep, bf16_ulp_distance, check_output, f64
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("layer", [0, 27])
+@pytest.mark.parametrize("layer", [0, 13, 27])
 def test_streaming_episode_sampled_steps(layer):
     if not torch.cuda.is_available():
         pytest.skip("needs a CUDA device")
@@ -29,14 +29,14 @@ def test_streaming_episode_sampled_steps(layer):
             L, n = cfg.call(s)
             x = W.make_new_tokens(cfg.step_config(s, layer))
             g = gs.step(L, x["q_new"], x["k_new"], x["v_new"])
-            # oracle cache: rotate + round the new keys, copy the values
-            kc[L:L + n] = so.round_bf16(so.rope(f64(x["k_new"]), L, cfg.rope_theta))
-            vc[L:L + n] = f64(x["v_new"])
             if s in sampled:
-                q_rot = so.rope(f64(x["q_new"]), L, cfg.rope_theta)
-                for i in sorted({0, n // 2, n - 1}):
-                    o, l = so.attend_range(q_rot[i:i + 1], kc, vc, L + i, 0, L + i + 1)
-                    check_output("bf16", g["out"][i:i + 1], g["lse"][i:i + 1], o, l)
+                # the oracle's step rotates, rounds and appends the new keys itself and attends all rows
+                r = so.step(f64(x["q_new"]), f64(x["k_new"]), f64(x["v_new"]), kc, vc, L, cfg.rope_theta, storage="bf16")
+                check_output("bf16", g["out"], g["lse"], r["out"], r["lse"])
+            else:
+                # oracle cache only: rotate + round the new keys, copy the values
+                kc[L:L + n] = so.round_bf16(so.rope(f64(x["k_new"]), L, cfg.rope_theta))
+                vc[L:L + n] = f64(x["v_new"])
         assert L + n == T
         assert bf16_ulp_distance(gs.k_cache.permute(1, 0, 2), kc).max() <= 1
         assert np.array_equal(f64(gs.v_cache.permute(1, 0, 2)), vc)

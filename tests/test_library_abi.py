@@ -31,11 +31,35 @@ def test_every_declared_symbol_is_exported(lib):
     assert sorted(B.EXPORTS) == names
 
 
-def test_struct_sizes_match_the_header_layout():
-    # 9 ints + float + double after a size_t: no hidden padding surprises on LP64
-    assert ctypes.sizeof(B.evlnStepParams) == 56
-    assert ctypes.sizeof(B.evlnPagedParams) == 56
-    assert ctypes.sizeof(B.evlnGatherParams) == 40
+def test_struct_sizes_match_the_header_layout(tmp_path):
+    # what the C compiler makes of include/evln.h is what the ctypes structures must be
+    import subprocess
+    src = tmp_path / "sizes.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "evln.h"\n'
+                   'int main(void) { printf("%zu %zu %zu %zu %zu\\n", sizeof(evlnStepParams), sizeof(evlnPagedParams), '
+                   'sizeof(evlnGatherParams), offsetof(evlnStepParams, rope_table), offsetof(evlnGatherParams, rope_table)); '
+                   'return 0; }\n')
+    exe = tmp_path / "sizes"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
+    step, paged, gather, off_step, off_gather = map(int, subprocess.check_output([str(exe)]).split())
+    assert ctypes.sizeof(B.evlnStepParams) == step == 72
+    assert ctypes.sizeof(B.evlnPagedParams) == paged == 56
+    assert ctypes.sizeof(B.evlnGatherParams) == gather == 56
+    assert B.evlnStepParams.rope_table.offset == off_step
+    assert B.evlnGatherParams.rope_table.offset == off_gather
+
+
+def test_page_table_check_on_the_host(lib):
+    # no GPU involved: range, duplicates within and across episodes, short tables
+    p = B.paged_params(28, 4, 128, 2, 64, 16, 8, 1e6)
+    ok = [[0, 1, 9, 9, 9, 9, 9, 9], [2, 3, 9, 9, 9, 9, 9, 9]]           # entries past the needed pages are ignored
+    assert B.evlnPagedCheckTable(p, [100, 70], [0, 10, 20], ok) == (B.EVLN_OK, -1, -1)
+    assert B.evlnPagedCheckTable(p, [100, 70], [0, 10, 20], [[0, 1] + [9] * 6, [2, 1] + [9] * 6]) == (B.EVLN_INVALID_VALUE, 1, 1)
+    assert B.evlnPagedCheckTable(p, [100, 70], [0, 10, 20], [[0, 0] + [9] * 6, [2, 3] + [9] * 6]) == (B.EVLN_INVALID_VALUE, 0, 1)
+    assert B.evlnPagedCheckTable(p, [100, 70], [0, 10, 20], [[0, 16] + [9] * 6, [2, 3] + [9] * 6]) == (B.EVLN_INVALID_VALUE, 0, 1)
+    assert B.evlnPagedCheckTable(p, [100, 70], [0, 10, 20], [[0, -1] + [9] * 6, [2, 3] + [9] * 6]) == (B.EVLN_INVALID_VALUE, 0, 1)
+    assert B.evlnPagedCheckTable(p, [600, 70], [0, 10, 20], ok)[0] == B.EVLN_CACHE_FULL      # 10 pages needed, 8 per row
+    assert B.evlnRopeTableBytes(128, 196) == 196 * 64 * 16 and B.evlnRopeTableBytes(96, 4) == 0
 
 
 def test_error_strings(lib):

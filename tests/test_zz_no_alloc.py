@@ -6,8 +6,11 @@ their control loop), so they can create neither a handle nor a workspace.
 evlnStepAttentionNoAlloc serves them from a scratch array inside the library.  Here it is
 called twice in a row through the C-ABI, on different inputs, and each result is compared with
 the handle + caller-workspace path within the tolerance of the other parity tests (the second
-call also shows that what the first left in the shared scratch does no harm).  Collected last
-on purpose, so that a run stopping at the first failure has already run everything else.
+call also shows that what the first left in the shared scratch does no harm), and with the fp64
+oracle on the same inputs, so that the two CUDA paths cannot agree on a wrong answer.  The status
+word of the allocation-free path (read through evlnGetDeviceStatus without a handle) must stay
+clear.  Collected last on purpose, so that a run stopping at the first failure has already run
+everything else.
 """
 import dataclasses
 
@@ -16,6 +19,7 @@ import torch
 
 from paper_2512_10310_b200 import binding as B
 from paper_2512_10310_b200 import workloads as W
+from tests.helpers import check_output, oracle_step
 
 pytestmark = pytest.mark.gpu
 
@@ -62,6 +66,10 @@ def test_no_alloc_matches_regular_path_twice():
             rel = (out.float() - ref_out.float()).norm() / ref_out.float().norm()
             assert rel.item() <= 1e-2
             assert (lse - ref_lse).abs().max().item() <= 1e-3
+            assert B.evlnGetDeviceStatus(None) == 0, "a kernel of the allocation-free call gave up on a bounded wait"
+            r = oracle_step("bf16", x["k_cache"], x["v_cache"], x["q_new"], x["k_new"], x["v_new"], L, cfg.rope_theta)
+            check_output("bf16", out, lse, r["out"], r["lse"])
+            check_output("bf16", ref_out, ref_lse, r["out"], r["lse"])
     finally:
         B.evlnDestroy(handle)
 
