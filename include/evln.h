@@ -228,6 +228,52 @@ evlnStatus_t evlnPagedCheckTable(const evlnPagedParams* params, const int* h_cac
                                  const int* h_new_offsets, const int* h_page_table,
                                  int* h_bad_episode, int* h_bad_index);
 
+/* ---- packed sequence under the action-isolating mask (Sec. 3.3, packed training via action
+ *      isolation; forward pass only) -----------------------------------------------------------
+ *
+ * A packed sequence is  I, v_1, a_1, v_2, a_2, ..., v_N, a_N : instr_len instruction tokens, then
+ * N frames of frame_tokens visual tokens, each followed by its chunk of action_tokens action
+ * tokens.  Under the mask of Sec. 3.3 a visual (or instruction) token attends causally to the
+ * instruction and the visual tokens up to itself, never to an action token; an action token of
+ * chunk t attends to the instruction, to v_1 .. v_t and to its own chunk up to itself, never to
+ * another chunk.  Position ids (the paper does not print them): the instruction and the visual
+ * tokens are numbered contiguously as if no action token were there, chunk t continues after v_t.
+ *
+ * evlnPackedForward runs the whole sequence in one call and six launches, whatever N is: the
+ * instruction and visual rows as ONE causal step on an empty cache (a query tile never loads a
+ * KV tile beyond its own last token, and action tokens are not among its keys at all), then all
+ * N action chunks as ONE batch whose items share prefixes of the cache just written and keep
+ * their own rotated keys / values in a separate buffer.  No mask operand exists: the blocks the
+ * mask removes are never loaded.
+ *   q [T, Hq, D], k, v [T, Hkv, D]: the packed sequence, T = instr_len + N (frame_tokens +
+ *       action_tokens), token strides in elements (multiples of 8);
+ *   k_cache, v_cache [Hkv, cache_capacity, D]: receive the rotated keys and the values of the
+ *       instruction + visual tokens at slots 0 .. instr_len + N frame_tokens - 1 (the cache an
+ *       inference run over the same frames would hold); EVLN_CACHE_FULL if they do not fit;
+ *   workspace: evlnPackedWorkspaceSize bytes (rotated queries, the chunks' keys/values, split partials);
+ *   out [T, Hq, D], lse_out [T, Hq] or NULL: rows in the order of the packed sequence.
+ * bf16, head_dim 128, at most 256 frames; otherwise EVLN_NOT_SUPPORTED.                         */
+typedef struct {
+    size_t struct_size;      /* sizeof(evlnPackedParams)                                     */
+    int dtype;               /* EVLN_BF16                                                    */
+    int num_q_heads, num_kv_heads, head_dim;
+    int instr_len;           /* |I|                                                          */
+    int frame_tokens;        /* |v|                                                          */
+    int action_tokens;       /* |a|                                                          */
+    int num_frames;          /* N                                                            */
+    int cache_capacity;      /* token slots per kv head in k_cache / v_cache                 */
+    int kv_chunk_tiles;      /* max 128-key tiles per work item of the action batch; 0 = heuristic */
+    float softmax_scale;     /* 0 -> 1/sqrt(D)                                               */
+    double rope_theta;
+} evlnPackedParams;
+
+evlnStatus_t evlnPackedWorkspaceSize(evlnHandle_t handle, const evlnPackedParams* params, size_t* bytes);
+evlnStatus_t evlnPackedForward(evlnHandle_t handle, const evlnPackedParams* params,
+                               const void* q, const void* k, const void* v,
+                               long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                               void* k_cache, void* v_cache, void* workspace, size_t workspace_bytes,
+                               void* out, float* lse_out, void* stream);
+
 /* ---- allocation-free variant ------------------------------------------------------------ */
 
 /* Largest split workspace the allocation-free call can serve (bytes of its built-in scratch). */

@@ -31,6 +31,7 @@ EXPORTS = [
     "evlnRopeAppend", "evlnStepAttention", "evlnStepCombine", "evlnStep",
     "evlnPagedWorkspaceSize", "evlnPagedRopeAppend", "evlnPagedStepAttention", "evlnPagedStepCombine",
     "evlnPagedCheckTable",
+    "evlnPackedWorkspaceSize", "evlnPackedForward",
     "evlnStepAttentionNoAlloc",
     "evlnSampleFrames", "evlnStoreAppend", "evlnGatherRope", "evlnStoreOffload", "evlnStoreFetch",
 ]
@@ -51,6 +52,13 @@ class evlnPagedParams(Structure):
                 ("num_kv_heads", c_int), ("head_dim", c_int), ("batch", c_int),
                 ("page_size", c_int), ("num_pages", c_int), ("max_pages_per_seq", c_int),
                 ("kv_chunk_tiles", c_int), ("softmax_scale", c_float), ("rope_theta", c_double)]
+
+
+class evlnPackedParams(Structure):
+    _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_q_heads", c_int), ("num_kv_heads", c_int),
+                ("head_dim", c_int), ("instr_len", c_int), ("frame_tokens", c_int), ("action_tokens", c_int),
+                ("num_frames", c_int), ("cache_capacity", c_int), ("kv_chunk_tiles", c_int),
+                ("softmax_scale", c_float), ("rope_theta", c_double)]
 
 
 class evlnGatherParams(Structure):
@@ -127,6 +135,10 @@ def lib():
                                              c_void_p, c_size_t, c_void_p]
         L.evlnPagedStepCombine.argtypes = [c_void_p, gp, c_void_p, ip, ip, c_void_p, c_void_p, c_void_p]
         L.evlnPagedCheckTable.argtypes = [gp, ip, ip, ip, ip, ip]
+        kp = POINTER(evlnPackedParams)
+        L.evlnPackedWorkspaceSize.argtypes = [c_void_p, kp, POINTER(c_size_t)]
+        L.evlnPackedForward.argtypes = [c_void_p, kp, c_void_p, c_void_p, c_void_p, c_long, c_long, c_long, c_void_p,
+                                        c_void_p, c_void_p, c_size_t, c_void_p, c_void_p, c_void_p]
         L.evlnStepAttentionNoAlloc.argtypes = [pp, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         qp = POINTER(evlnGatherParams)
         L.evlnSampleFrames.argtypes = [c_int, c_int, c_int, c_int, POINTER(c_int)]
@@ -329,6 +341,27 @@ def evlnPagedStepCombine(handle, params, workspace, cache_lens, new_offsets, out
     _check(lib().evlnPagedStepCombine(handle, byref(params), _ptr(workspace), _ints(cache_lens),
                                       _ints(new_offsets), _ptr(out), _ptr(lse_out), _stream(stream)),
            "evlnPagedStepCombine")
+
+
+def packed_params(num_q_heads, num_kv_heads, head_dim, instr_len, frame_tokens, action_tokens, num_frames,
+                  cache_capacity, rope_theta, softmax_scale=0.0, kv_chunk_tiles=0, dtype=EVLN_BF16) -> evlnPackedParams:
+    return evlnPackedParams(ctypes.sizeof(evlnPackedParams), dtype, num_q_heads, num_kv_heads, head_dim, instr_len,
+                            frame_tokens, action_tokens, num_frames, cache_capacity, kv_chunk_tiles, softmax_scale,
+                            rope_theta)
+
+
+def evlnPackedWorkspaceSize(handle, params) -> int:
+    v = c_size_t(0)
+    _check(lib().evlnPackedWorkspaceSize(handle, byref(params), byref(v)), "evlnPackedWorkspaceSize")
+    return int(v.value)
+
+
+def evlnPackedForward(handle, params, q, k, v, k_cache, v_cache, workspace, out, lse_out=None, stream=None):
+    """A packed sequence I, v_1, a_1, ..., v_N, a_N under the action-isolating mask, in one call."""
+    _check(lib().evlnPackedForward(handle, byref(params), _ptr(q), _ptr(k), _ptr(v), int(q.stride(0)), int(k.stride(0)),
+                                   int(v.stride(0)), _ptr(k_cache), _ptr(v_cache), _ptr(workspace),
+                                   int(workspace.numel() * workspace.element_size()), _ptr(out), _ptr(lse_out),
+                                   _stream(stream)), "evlnPackedForward")
 
 
 def evlnStepAttentionNoAlloc(params, q_rot, k_cache, v_cache, out, lse_out=None, stream=None):

@@ -93,8 +93,8 @@ cudaError_t launch_pair_pdl(void (*kernel)(KArgs...), dim3 grid, size_t smem, cu
 bool attention_register_pool_ok()
 {
     cudaFuncAttributes fa;
-    const void* kernels[3] = {(const void*)attn_pair_kernel<false, NoLens>, (const void*)attn_pair_kernel<true, BatchLens>,
-                              (const void*)attn_solo_kernel};
+    const void* kernels[4] = {(const void*)attn_pair_kernel<false, NoLens>, (const void*)attn_pair_kernel<true, BatchLens>,
+                              (const void*)attn_solo_kernel, (const void*)attn_tail_kernel};
     for (const void* k : kernels) {
         if (cudaFuncGetAttributes(&fa, k) != cudaSuccess) return false;
         if (fa.numRegs != kRegsLaunch) return false;
@@ -404,6 +404,8 @@ evlnStatus_t evlnCreate(evlnHandle_t* handle, int device)
                                  kTcSmemBytes);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(attn_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSoloSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
     if (e == cudaSuccess && !attention_register_pool_ok()) {
         cudaFree(h->d_status);
         delete h;
@@ -524,9 +526,9 @@ evlnStatus_t evlnStepQRotSize(evlnHandle_t h, const evlnStepParams* p, size_t* b
     return EVLN_OK;
 }
 
-evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
-                            const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok,
-                            void* q_rot, void* k_cache, void* v_cache, void* stream)
+static evlnStatus_t rope_append_impl(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
+                                     const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                                     void* q_rot, void* k_cache, void* v_cache, void* stream, const PackedMap& map)
 {
     evlnStatus_t s = check_step_params(h, p);
     if (s != EVLN_OK) return s;
@@ -552,6 +554,7 @@ evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void*
     a.log2_theta = log2(p->rope_theta);
     a.table = (const double2*)p->rope_table;
     a.table_first = p->rope_table_first_pos;
+    a.map = map;
     NoLens nl = {};
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16)
@@ -560,6 +563,14 @@ evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void*
         launch_pdl(rope_append_kernel<float, false, NoLens>, dim3(p->num_new), dim3(256), 0, st, a, nl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+evlnStatus_t evlnRopeAppend(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
+                            const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                            void* q_rot, void* k_cache, void* v_cache, void* stream)
+{
+    return rope_append_impl(h, p, q_new, k_new, v_new, q_stride_tok, k_stride_tok, v_stride_tok, q_rot, k_cache,
+                            v_cache, stream, PackedMap{0, 0, 0, 0});
 }
 
 evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const void* q_rot, const void* k_cache,
@@ -640,8 +651,8 @@ evlnStatus_t evlnStepAttention(evlnHandle_t h, const evlnStepParams* p, const vo
 }
 
 
-evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void* workspace, void* out,
-                             float* lse_out, void* stream)
+static evlnStatus_t step_combine_impl(evlnHandle_t h, const evlnStepParams* p, const void* workspace, void* out,
+                                      float* lse_out, void* stream, const PackedMap& map)
 {
     evlnStatus_t s = check_step_params(h, p);
     if (s != EVLN_OK) return s;
@@ -656,9 +667,16 @@ evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void
     a.lse_part = a.o_part + (size_t)S * p->num_kv_heads * R * p->head_dim;
     a.out = out; a.lse_out = lse_out;
     a.Hkv = p->num_kv_heads; a.G = G; a.D = p->head_dim; a.rows = R; a.num_splits = S;
+    a.map = map;
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16) return launch_combine<__nv_bfloat16>(h, a, p->head_dim, false, nullptr, st);
     return launch_combine<float>(h, a, p->head_dim, false, nullptr, st);
+}
+
+evlnStatus_t evlnStepCombine(evlnHandle_t h, const evlnStepParams* p, const void* workspace, void* out,
+                             float* lse_out, void* stream)
+{
+    return step_combine_impl(h, p, workspace, out, lse_out, stream, PackedMap{0, 0, 0, 0});
 }
 
 evlnStatus_t evlnStep(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
@@ -833,6 +851,184 @@ evlnStatus_t evlnPagedCheckTable(const evlnPagedParams* p, const int* h_cache_le
 }
 
 }  // extern "C"
+
+// ---- packed sequence under the action-isolating mask (Sec. 3.3) -----------------------------
+
+namespace {
+struct PackedPlan {
+    int n_vis, n_act;            // instruction + visual tokens; action tokens
+    evlnStepParams vis;          // the visual run as one step on an empty cache
+    int lens[kMaxBatch];         // per action chunk: visible prefix of the cache
+    int offs[kMaxBatch + 1];     // per action chunk: first own token
+    int chunk, smax;             // KV tiles per work item of the action batch, its largest split count
+    long items;
+    size_t off_qv, off_qa, off_tk, off_tv, off_part, bytes;   // workspace layout
+};
+
+evlnStatus_t plan_packed(evlnHandle_t h, const evlnPackedParams* p, PackedPlan* pl)
+{
+    if (!h || !p) return EVLN_INVALID_VALUE;
+    if (p->struct_size != sizeof(evlnPackedParams)) return EVLN_INVALID_VALUE;
+    if (p->num_q_heads <= 0 || p->num_kv_heads <= 0 || p->num_q_heads % p->num_kv_heads != 0) return EVLN_INVALID_VALUE;
+    if (p->instr_len < 0 || p->frame_tokens < 0 || p->action_tokens < 0 || p->num_frames < 0 || p->kv_chunk_tiles < 0)
+        return EVLN_INVALID_VALUE;
+    if (!(p->rope_theta > 0.0) || !(p->softmax_scale >= 0.f)) return EVLN_INVALID_VALUE;
+    if (p->dtype != EVLN_BF16 || p->head_dim != 128 || p->num_frames > kMaxBatch) return EVLN_NOT_SUPPORTED;
+    const long n_vis = (long)p->instr_len + (long)p->num_frames * p->frame_tokens;
+    const long n_act = (long)p->num_frames * p->action_tokens;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    if ((n_vis + n_act) * G > (1 << 24)) return EVLN_NOT_SUPPORTED;
+    if (n_vis > (long)p->cache_capacity) return EVLN_CACHE_FULL;
+    pl->n_vis = (int)n_vis;
+    pl->n_act = (int)n_act;
+    evlnStepParams& sp = pl->vis;
+    memset(&sp, 0, sizeof(sp));
+    sp.struct_size = sizeof(sp);
+    sp.dtype = EVLN_BF16;
+    sp.num_q_heads = p->num_q_heads; sp.num_kv_heads = p->num_kv_heads; sp.head_dim = 128;
+    sp.cache_len = 0; sp.num_new = (int)n_vis; sp.cache_capacity = p->cache_capacity;
+    sp.num_splits = 0; sp.kernel = EVLN_KERNEL_AUTO;
+    sp.softmax_scale = p->softmax_scale; sp.rope_theta = p->rope_theta;
+    for (int t = 0; t < p->num_frames; ++t) {
+        pl->lens[t] = p->instr_len + (t + 1) * p->frame_tokens;      // chunk t sees the instruction and v_1 .. v_{t+1}
+        pl->offs[t] = t * p->action_tokens;
+    }
+    pl->offs[p->num_frames] = (int)n_act;
+    pl->chunk = pl->smax = 1;
+    pl->items = 0;
+    if (n_act > 0)
+        batch_schedule(h->num_sms, G, p->num_kv_heads, p->num_frames, pl->lens, pl->offs, true, p->kv_chunk_tiles,
+                       &pl->chunk, &pl->smax, &pl->items);
+    size_t part_v = 0;
+    if (n_vis > 0) {
+        evlnStatus_t s = check_step_params(h, &sp);
+        if (s != EVLN_OK) return s;
+        part_v = partial_bytes(resolve_splits(h, &sp), p->num_kv_heads, n_vis * G, 128);
+    }
+    const size_t part_a = n_act > 0 ? partial_bytes(pl->smax, p->num_kv_heads, n_act * G, 128) : 0;
+    size_t off = 0;
+    pl->off_qv = off; off += round_up((size_t)n_vis * p->num_q_heads * 128 * 2, 256);
+    pl->off_qa = off; off += round_up((size_t)n_act * p->num_q_heads * 128 * 2, 256);
+    pl->off_tk = off; off += round_up((size_t)n_act * p->num_kv_heads * 128 * 2, 256);
+    pl->off_tv = off; off += round_up((size_t)n_act * p->num_kv_heads * 128 * 2, 256);
+    pl->off_part = off; off += part_v > part_a ? part_v : part_a;
+    pl->bytes = off > 256 ? off : 256;
+    return EVLN_OK;
+}
+}  // namespace
+
+extern "C" evlnStatus_t evlnPackedWorkspaceSize(evlnHandle_t h, const evlnPackedParams* p, size_t* bytes)
+{
+    PackedPlan pl;
+    evlnStatus_t s = plan_packed(h, p, &pl);
+    if (s != EVLN_OK) return s;
+    if (!bytes) return EVLN_INVALID_VALUE;
+    *bytes = pl.bytes;
+    return EVLN_OK;
+}
+
+extern "C" evlnStatus_t evlnPackedForward(evlnHandle_t h, const evlnPackedParams* p, const void* q, const void* k,
+                                          const void* v, long q_stride_tok, long k_stride_tok, long v_stride_tok,
+                                          void* k_cache, void* v_cache, void* workspace, size_t workspace_bytes,
+                                          void* out, float* lse_out, void* stream)
+{
+    PackedPlan pl;
+    evlnStatus_t s = plan_packed(h, p, &pl);
+    if (s != EVLN_OK) return s;
+    if (pl.n_vis + pl.n_act == 0) return EVLN_OK;
+    if (!q || !k || !v || !k_cache || !v_cache || !workspace || !out) return EVLN_INVALID_VALUE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache) ||
+        !aligned16(workspace) || !aligned16(out))
+        return EVLN_INVALID_VALUE;
+    if (q_stride_tok < (long)p->num_q_heads * 128 || k_stride_tok < (long)p->num_kv_heads * 128 ||
+        v_stride_tok < (long)p->num_kv_heads * 128 || q_stride_tok % 8 || k_stride_tok % 8 || v_stride_tok % 8)
+        return EVLN_INVALID_VALUE;
+    if (workspace_bytes < pl.bytes) return EVLN_WORKSPACE_TOO_SMALL;
+    if (!device_is_current(h)) return EVLN_INVALID_VALUE;
+    char* ws = (char*)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const PackedMap map_v{p->instr_len, p->frame_tokens, p->action_tokens, 0};
+    const PackedMap map_a{p->instr_len, p->frame_tokens, p->action_tokens, 1};
+
+    // the instruction and the visual tokens: ONE causal step on an empty cache; its query tiles never
+    // load a KV tile past their own last token, and no action token is among the keys at all
+    if (pl.n_vis > 0) {
+        s = rope_append_impl(h, &pl.vis, q, k, v, q_stride_tok, k_stride_tok, v_stride_tok, ws + pl.off_qv, k_cache, v_cache,
+                             stream, map_v);
+        if (s != EVLN_OK) return s;
+        const size_t part_v = partial_bytes(resolve_splits(h, &pl.vis), p->num_kv_heads, (long)pl.n_vis * G, 128);
+        s = evlnStepAttention(h, &pl.vis, ws + pl.off_qv, k_cache, v_cache, ws + pl.off_part, part_v, stream);
+        if (s != EVLN_OK) return s;
+        s = step_combine_impl(h, &pl.vis, ws + pl.off_part, out, lse_out, stream, map_v);
+        if (s != EVLN_OK) return s;
+    }
+    if (pl.n_act == 0) return EVLN_OK;
+
+    // all action chunks in one batch: chunk t sees the first lens[t] tokens of the cache just written
+    // and its own tokens, which live in a buffer of their own (nobody else's keys)
+    BatchLens bl;
+    fill_batch_lens(&bl, G, p->num_kv_heads, p->num_frames, pl.lens, pl.offs, pl.chunk, true);
+    if (bl.item_off[p->num_frames] != (int)pl.items || pl.items <= 0 || pl.items > 0x3fffffffL) return EVLN_NOT_SUPPORTED;
+    {
+        RopeArgs a = {};
+        a.q_new = q; a.k_new = k; a.v_new = v;
+        a.q_rot = ws + pl.off_qa; a.k_cache = ws + pl.off_tk; a.v_cache = ws + pl.off_tv; a.page_table = nullptr;
+        a.q_stride = q_stride_tok; a.k_stride = k_stride_tok; a.v_stride = v_stride_tok;
+        a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = 128;
+        a.num_new = pl.n_act; a.batch = p->num_frames; a.page_size = 1; a.max_pages = 0;
+        a.log2_theta = log2(p->rope_theta);
+        a.tail = 1;
+        a.map = map_a;
+        launch_pdl(rope_append_kernel<__nv_bfloat16, true, BatchLens>, dim3(pl.n_act), dim3(256), 0, st, a, bl);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    const long rows = (long)pl.n_act * G;
+    {
+        CUtensorMap tm_q, tm_k, tm_v, tm_kt, tm_vt;
+        cuuint32_t box_q[3] = {64, 128, 1}, box_k[3] = {64, 64, 1}, box_v[3] = {64, 128, 1};
+        {
+            cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)p->num_kv_heads};
+            cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
+            if (!encode_map(h, &tm_q, ws + pl.off_qa, 3, dims, strides, box_q)) return EVLN_INVALID_VALUE;
+        }
+        {
+            cuuint64_t dims[3] = {128, (cuuint64_t)pl.n_vis, (cuuint64_t)p->num_kv_heads};
+            cuuint64_t strides[2] = {256, (cuuint64_t)p->cache_capacity * 256};
+            if (!encode_map(h, &tm_k, k_cache, 3, dims, strides, box_k)) return EVLN_INVALID_VALUE;
+            if (!encode_map(h, &tm_v, v_cache, 3, dims, strides, box_v)) return EVLN_INVALID_VALUE;
+        }
+        {
+            cuuint64_t dims[3] = {128, (cuuint64_t)pl.n_act, (cuuint64_t)p->num_kv_heads};
+            cuuint64_t strides[2] = {256, (cuuint64_t)pl.n_act * 256};
+            if (!encode_map(h, &tm_kt, ws + pl.off_tk, 3, dims, strides, box_k)) return EVLN_INVALID_VALUE;
+            if (!encode_map(h, &tm_vt, ws + pl.off_tv, 3, dims, strides, box_v)) return EVLN_INVALID_VALUE;
+        }
+        const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf(128.f);
+        TcAttnArgs a = {};
+        a.o_part = (float*)(ws + pl.off_part);
+        a.lse_part = a.o_part + (size_t)pl.smax * p->num_kv_heads * rows * 128;
+        a.page_table = nullptr; a.status = h->d_status;
+        a.Hkv = p->num_kv_heads; a.G = G; a.rows = (int)rows;
+        a.batch = p->num_frames; a.max_pages = 0; a.chunk_tiles = pl.chunk;
+        a.scale_log2 = scale * 1.4426950408889634f;
+        a.div_g = make_fast_div((uint32_t)G);
+        a.div_s = make_fast_div(1u);
+        launch_pair_pdl(attn_tail_kernel, dim3(2 * (int)pl.items), kTcSmemBytes, st, tm_q, tm_k, tm_v, tm_kt, tm_vt, a, bl);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    CombineArgs c = {};
+    c.o_part = (const float*)(ws + pl.off_part);
+    c.lse_part = c.o_part + (size_t)pl.smax * p->num_kv_heads * rows * 128;
+    c.out = out; c.lse_out = lse_out;
+    c.Hkv = p->num_kv_heads; c.G = G; c.D = 128; c.rows = (int)rows; c.num_splits = pl.smax;
+    c.batch = p->num_frames; c.unit_rows = kUnitRows; c.chunk_tiles = pl.chunk;
+    c.tail = 1;
+    c.map = map_a;
+    return launch_combine<__nv_bfloat16>(h, c, 128, true, &bl, st);
+}
 
 // ---- un-rotated store + frame sampler ------------------------------------------------------
 
