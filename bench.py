@@ -345,6 +345,211 @@ def ring_layers_for(kv_bytes):
     return max(2, min(RING_LAYERS, int(2.2 * L2_BYTES / kv_bytes) + 1))
 
 
+def graph_of(fn):
+    """A CUDA graph of one call of fn() (warmed once on a side stream first)."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        fn()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g
+
+
+def measure_widening(B, handle, cfg, dev, barrier, peaks):
+    """The workloads beyond the plain step (7B-class layer shape throughout):
+    a packed sequence under the action-isolating mask, one call against the loop of 2N+1 steps;
+    the un-rotated store re-indexed by a frame sampler (gather + rotate pass, then the step);
+    reloads of frame segments from a pinned host store, alone and beside the attention of a step."""
+    Hq, Hkv, D, theta = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim, cfg.rope_theta
+    bf = torch.bfloat16
+    gen = torch.Generator(device=dev).manual_seed(99)
+    mk = lambda *sh: (torch.randn(*sh, generator=gen, device=dev, dtype=torch.float32) * cfg.input_scale).to(bf)
+    res = {}
+
+    # ---- packed sequence: instruction 256, 12 frames of 196 visual + 8 action tokens ----
+    I, F, A, N = 256, 196, 8, 12
+    T, n_vis = I + N * (F + A), I + N * F
+    pp = B.packed_params(Hq, Hkv, D, I, F, A, N, n_vis, theta)
+    reps = 8                      # independent copies cycled through, so that the caches do not sit in L2
+    packs = [dict(q=mk(T, Hq, D), k=mk(T, Hkv, D), v=mk(T, Hkv, D), kc=torch.empty((Hkv, n_vis + A, D), dtype=bf, device=dev),
+                  vc=torch.empty((Hkv, n_vis + A, D), dtype=bf, device=dev),
+                  ws=torch.empty(B.evlnPackedWorkspaceSize(handle, pp), dtype=torch.uint8, device=dev),
+                  out=torch.empty((T, Hq, D), dtype=bf, device=dev)) for _ in range(reps)]
+    pp = B.packed_params(Hq, Hkv, D, I, F, A, N, n_vis + A, theta)
+
+    def packed_all():
+        for y in packs:
+            B.evlnPackedForward(handle, pp, y["q"], y["k"], y["v"], y["kc"], y["vc"], y["ws"], y["out"])
+
+    # the same rows through ordinary steps: the instruction, then frame step + action step per frame
+    calls = [(0, I, 0)]
+    for t in range(N):
+        r0 = I + t * (F + A)
+        calls += [(I + t * F, F, r0), (I + (t + 1) * F, A, r0 + F)]
+    sp = [B.step_params("bf16", Hq, Hkv, D, L, n, n_vis + A, theta) for L, n, _ in calls]
+    qr = torch.empty(max(B.evlnStepQRotSize(handle, p) for p in sp), dtype=torch.uint8, device=dev)
+    wl = torch.empty(max(B.evlnStepWorkspaceSize(handle, p) for p in sp), dtype=torch.uint8, device=dev)
+
+    def loop_all():
+        for y in packs:
+            for p, (L, n, r0) in zip(sp, calls):
+                B.evlnStep(handle, p, y["q"][r0:r0 + n], y["k"][r0:r0 + n], y["v"][r0:r0 + n], qr, y["kc"], y["vc"], wl,
+                           y["out"][r0:r0 + n])
+
+    g1, g2 = graph_of(packed_all), graph_of(loop_all)
+    t1 = timed_replays(g1, MIN_REPLAYS, reps, barrier)
+    t2 = timed_replays(g2, MIN_REPLAYS, reps, barrier)
+    kind_flops = 4 * D * Hq * (n_vis * (n_vis + 1) // 2 + sum(A * (I + (t + 1) * F) + A * (A + 1) // 2 for t in range(N)))
+    res["packed_forward"] = {
+        "workload": f"packed sequence: instruction {I}, {N} frames x ({F} visual + {A} action tokens), {T} tokens",
+        "one_call_us": r3(t1["median"]), "one_call_p10": r3(t1["p10"]), "one_call_p90": r3(t1["p90"]), "launches_one_call": 6,
+        "step_loop_us": r3(t2["median"]), "launches_step_loop": 3 * len(calls), "speedup": round(t2["median"] / t1["median"], 2),
+        "tflops_one_call": round(kind_flops / t1["median"] / 1e6, 1)}
+    del g1, g2, packs
+    torch.cuda.empty_cache()
+
+    # ---- un-rotated store + frame sampler: 16 kept frames of 196 tokens + instruction 256 -> 3392 kept tokens ----
+    kept_frames, store_frames = 16, 64
+    kept = I + kept_frames * F
+    store_cap = I + store_frames * F
+    layers = ring_layers_for(2 * kept * Hkv * D * 2)
+    tbl = torch.empty(B.evlnRopeTableBytes(D, kept + F), dtype=torch.uint8, device=dev)
+    B.evlnRopeTable(handle, D, theta, 0, kept + F, tbl)
+    gp = B.gather_params("bf16", Hkv, D, store_cap, kept + F, theta, rope_table=tbl, rope_table_first_pos=0,
+                         rope_table_count=kept + F)
+    frames = B.evlnSampleFrames(B.EVLN_SAMPLE_UNIFORM, store_frames, kept_frames)
+    seg_src = [0] + [I + f * F for f in frames]
+    seg_len = [I] + [F] * kept_frames
+    st_p = B.step_params("bf16", Hq, Hkv, D, kept, F, kept + F, theta, rope_table=tbl, rope_table_first_pos=0,
+                         rope_table_count=kept + F)
+    lay = [dict(ks=mk(Hkv, store_cap, D), vs=mk(Hkv, store_cap, D), kw=torch.empty((Hkv, kept + F, D), dtype=bf, device=dev),
+                vw=torch.empty((Hkv, kept + F, D), dtype=bf, device=dev), q=mk(F, Hq, D), k=mk(F, Hkv, D), v=mk(F, Hkv, D),
+                qr=torch.empty(B.evlnStepQRotSize(handle, st_p), dtype=torch.uint8, device=dev),
+                ws=torch.empty(B.evlnStepWorkspaceSize(handle, st_p), dtype=torch.uint8, device=dev),
+                out=torch.empty((F, Hq, D), dtype=bf, device=dev)) for _ in range(layers)]
+
+    def gather_all():
+        for y in lay:
+            B.evlnGatherRope(handle, gp, seg_src, seg_len, y["ks"], y["vs"], y["kw"], y["vw"])
+
+    def step_all():
+        for y in lay:
+            B.evlnStep(handle, st_p, y["q"], y["k"], y["v"], y["qr"], y["kw"], y["vw"], y["ws"], y["out"])
+
+    def both_all():
+        for y in lay:
+            B.evlnGatherRope(handle, gp, seg_src, seg_len, y["ks"], y["vs"], y["kw"], y["vw"])
+            B.evlnStep(handle, st_p, y["q"], y["k"], y["v"], y["qr"], y["kw"], y["vw"], y["ws"], y["out"])
+
+    tg = timed_replays(graph_of(gather_all), MIN_REPLAYS, layers, barrier)
+    ts = timed_replays(graph_of(step_all), MIN_REPLAYS, layers, barrier)
+    tb = timed_replays(graph_of(both_all), MIN_REPLAYS, layers, barrier)
+    moved = 2 * 2 * kept * Hkv * D * 2          # K and V of every kept token, read + written
+    res["reindexed_store"] = {
+        "workload": f"un-rotated store of {store_frames} frames, uniform sampler keeps {kept_frames}: {kept} kept tokens + {F} new",
+        "gather_rope_us": r3(tg["median"]), "gather_bytes": moved,
+        "gather_gbs": round(moved / tg["median"] / 1e3, 1), "gather_hbm_frac": round(moved / tg["median"] / 1e3 / peaks["hbm_gbs"], 4),
+        "step_us": r3(ts["median"]), "gather_plus_step_us": r3(tb["median"]), "ring_layers": layers}
+    del lay
+    torch.cuda.empty_cache()
+
+    # ---- host-resident store: reload of 1 and of 8 (= half of a budget of 16) frame segments for all 28
+    #      layers on a side stream, alone and beside the attention steps of those layers ----
+    L28 = 28
+    host_frames = 17
+    hk = [torch.empty((Hkv, host_frames * F, D), dtype=bf).pin_memory() for _ in range(2)]     # K and V host stores of one layer
+    ring = LayerRing(B, handle, cfg, dev, L28)
+    gpl = B.gather_params("bf16", Hkv, D, 16 * F, 16 * F, theta)
+    stores = [(torch.empty((Hkv, 16 * F, D), dtype=bf, device=dev), torch.empty((Hkv, 16 * F, D), dtype=bf, device=dev))
+              for _ in range(L28)]
+    side = torch.cuda.Stream()
+
+    def fetch(nseg):
+        for ks, vs in stores:
+            for sgi in range(nseg):
+                B.evlnStoreFetch(handle, gpl, hk[0], hk[1], sgi * F, F, ks, vs, sgi * F, stream=side)
+
+    def steps28():
+        for l in range(L28):
+            ring.step(l)
+
+    def wall_us(fn, reps=20):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        cur = torch.cuda.current_stream()
+        e0.record()
+        for _ in range(reps):
+            fn()
+            cur.wait_stream(side)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps
+
+    def with_side(nseg):
+        def f():
+            side.wait_stream(torch.cuda.current_stream())
+            fetch(nseg)
+            steps28()
+        return f
+
+    def fetch_only(nseg):
+        def f():
+            side.wait_stream(torch.cuda.current_stream())
+            fetch(nseg)
+        return f
+
+    t_steps = wall_us(steps28)
+    rec = {"workload": f"28 layers, frame segments of {F} tokens ({2 * F * Hkv * D * 2} bytes per layer and segment), pinned host store",
+           "steps_28_layers_us": r3(t_steps), "launch": "eager calls; copies on a side stream, the 28 layer-steps on the main stream"}
+    for nseg in (1, 8):
+        t_f = wall_us(fetch_only(nseg))
+        t_b = wall_us(with_side(nseg))
+        nbytes = nseg * L28 * 2 * F * Hkv * D * 2
+        rec[f"fetch_{nseg}_segments"] = {"bytes": nbytes, "alone_us": r3(t_f), "h2d_gbs": round(nbytes / t_f / 1e3, 1),
+                                          "beside_steps_us": r3(t_b), "exposed_us": r3(max(0.0, t_b - t_steps))}
+    res["host_store_fetch"] = rec
+    del ring, stores
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_profile_workload(args, local_rank):
+    """A few eager steps of ONE workload and nothing else: the small command that ncu captures are
+    taken on (launch lists and counter sets of single kernels).  Prints a short JSON line, no timing."""
+    from paper_2512_10310_b200 import binding as B
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    handle = B.evlnCreate(local_rank)
+    name = args.profile_workload
+    steps = max(1, args.steps)
+    if name == "paged_b4":
+        pc = dataclasses.replace(W.PAGED_B16, name="paged_b4", batch=4)
+        x = W.make_paged_inputs(pc)
+        pb = PagedBatch(B, handle, pc, x, dev, layers=1)
+        for _ in range(steps):
+            pb.step(0)
+        info = {"episodes": 4, "cache_lens": x["cache_lens"]}
+    else:
+        c = {"step_7b": W.STEP_7B, "long_70b": W.LONG_70B,
+             "action_7b": dataclasses.replace(W.STEP_7B, name="action_7b_L20656", cache_len=20656, num_new=8)}[name]
+        kv_bytes = 2 * (c.cache_len + c.num_new) * c.num_kv_heads * c.head_dim * 2
+        layers = 2 if kv_bytes > 64e6 else min(RING_LAYERS, ring_layers_for(kv_bytes))
+        ring = LayerRing(B, handle, c, dev, layers)
+        for i in range(steps):
+            ring.step(i % layers)
+        info = {"cache_len": c.cache_len, "new_tokens": c.num_new, "kv_splits": ring.splits, "ring_layers": layers}
+    torch.cuda.synchronize()
+    assert B.evlnGetDeviceStatus(handle) == 0
+    B.evlnDestroy(handle)
+    print(json.dumps({"profiled": name, "steps": steps, **info}), flush=True)
+
+
 def run_ours(args, rank, world, local_rank, dist):
     from paper_2512_10310_b200 import binding as B
 
@@ -403,7 +608,7 @@ def run_ours(args, rank, world, local_rank, dist):
     ring_mib = RING_LAYERS * ring.bytes_per_layer / 2 ** 20
     headline_splits = ring.splits
 
-    by_len, action_steps, by_config = [], [], []
+    by_len, action_steps, by_config, widening = [], [], [], None
     if world == 1 and not args.no_sweep:
         del g_step, g_attn, g_k1, g_k3, g_e2e
         ring.layers.clear()
@@ -476,6 +681,7 @@ def run_ours(args, rank, world, local_rank, dist):
         if not args.no_cpu_baseline:
             dt, _ = cpu_baseline_full_step(W.LONG_70B, reps=1)
             by_config[-2]["oracle_s"] = round(dt, 2)
+        widening = measure_widening(B, handle, cfg, dev, barrier, peaks)
         assert B.evlnGetDeviceStatus(handle) == 0, "a kernel gave up on a bounded wait"
     clocks = sampler.stop()
     B.evlnDestroy(handle)
@@ -536,6 +742,8 @@ def run_ours(args, rank, world, local_rank, dist):
         line["by_config"] = by_config
     if action_steps:
         line["action_token_step"] = action_steps
+    if widening:
+        line["widening"] = widening
     return line
 
 
@@ -625,12 +833,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads (cache-length sweep, by_config)")
+    ap.add_argument("--profile-workload", default=None, choices=["step_7b", "long_70b", "paged_b4", "action_7b"],
+                    help="run --steps eager steps of one workload and exit (the command ncu captures are taken on)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
+    if args.profile_workload:
+        if rank == 0:
+            run_profile_workload(args, local_rank)
+        return
     if args.impl == "reference":
         line = run_reference(args, rank, world)
         if line is not None:
