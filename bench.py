@@ -223,20 +223,23 @@ class LayerRing:
         with torch.cuda.stream(s_out if s_out is not None else cur):
             y["host_out"].copy_(y["out"], non_blocking=True)
 
-    def capture_e2e(self):
+    def capture_e2e(self, copy_streams=1):
         """One CUDA graph of a pass over the ring through the public calls with host buffers:
-        copies in on one stream, kernels on the capture stream, copies out on a third."""
-        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        copies in on side streams, kernels on the capture stream, copies out on further side
+        streams.  With more than one stream per direction consecutive steps' copies are independent
+        nodes of the graph, so a copy can be set up while the previous one still moves data."""
+        s_ins = [torch.cuda.Stream() for _ in range(copy_streams)]
+        s_outs = [torch.cuda.Stream() for _ in range(copy_streams)]
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             cur = torch.cuda.current_stream()
-            s_in.wait_stream(cur)
-            s_out.wait_stream(cur)
+            for s in s_ins + s_outs:
+                s.wait_stream(cur)
             self.make_table()
             for l in range(len(self.layers)):
-                self.step_e2e(l, s_in, s_out)
-            cur.wait_stream(s_in)
-            cur.wait_stream(s_out)
+                self.step_e2e(l, s_ins[l % copy_streams], s_outs[l % copy_streams])
+            for s in s_ins + s_outs:
+                cur.wait_stream(s)
         return g
 
 
