@@ -23,6 +23,9 @@ struct CombineArgs {
     // batches: per-episode split counts are derived from the lengths
     int batch, unit_rows, chunk_tiles;
     int tail;                // batch of items sharing a cache prefix (own tokens tiled separately)
+    FastDiv div_g;           // division by G, by the work-item size in KV tiles (chunk_tiles, at least 1):
+    FastDiv div_chunk;       //   a row's warp decodes its place with multiplications (an integer division costs
+                             //   as much as the rest of the merge)
     PackedMap map;           // where output token m goes (identity unless the call serves a packed sequence)
 };
 
@@ -34,13 +37,15 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
     asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long row = (long)blockIdx.x * 4 + warp;      // packed row within kv head
+    const uint32_t row = blockIdx.x * 4u + (uint32_t)warp;      // packed row within kv head (< 2^24, checked on the host)
     const int g = blockIdx.y;
-    if (row >= a.rows) return;
+    if (row >= (uint32_t)a.rows) return;
+    const uint32_t row_tok = fast_div(row, a.div_g);            // its token among the call's new tokens ...
+    const int row_head = (int)(row - row_tok * (uint32_t)a.G);  // ... and its query head within the group
 
     int S = a.num_splits;
     if (PAGED) {
-        const int tok = (int)(row / a.G);
+        const int tok = (int)row_tok;
         int lo = 0, hi = a.batch;
         while (hi - lo > 1) {
             int mid = (lo + hi) >> 1;
@@ -48,10 +53,11 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
         }
         const int b = lo;
         const int n_b = lens.new_off[b + 1] - lens.new_off[b];
-        const int local_row = (int)(row - (long)lens.new_off[b] * a.G);
-        const int unit = local_row / a.unit_rows;
-        S = ceil_div(a.tail ? tail_kv_tiles(lens.cache_len[b], n_b, a.G, unit, a.unit_rows)
-                            : unit_kv_tiles(lens.cache_len[b], n_b, a.G, unit, a.unit_rows), a.chunk_tiles);
+        const int local_row = (int)row - lens.new_off[b] * a.G;
+        const int unit = local_row / kUnitRows;                  // (a power of two)
+        const int nkv = a.tail ? tail_kv_tiles_fast(lens.cache_len[b], n_b, a.div_g, unit, kUnitRows)
+                               : unit_kv_tiles_fast(lens.cache_len[b], n_b, a.div_g, unit, kUnitRows);
+        S = (int)fast_div((uint32_t)(nkv + a.chunk_tiles - 1), a.div_chunk);
     }
 
     const long stride_s = (long)a.Hkv * a.rows;           // rows between consecutive splits
@@ -127,8 +133,8 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
     }
     const float inv = (wsum > 0.f) ? 1.f / wsum : 0.f;
 
-    const long tok = packed_row(a.map, row / a.G);
-    const int h = g * a.G + (int)(row % a.G);
+    const long tok = packed_row(a.map, (long)row_tok);
+    const int h = g * a.G + row_head;
     const int Hq = a.Hkv * a.G;
     T* dst = (T*)a.out + (tok * Hq + h) * D + lane * C;
 #pragma unroll

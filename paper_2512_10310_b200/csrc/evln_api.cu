@@ -330,9 +330,12 @@ void fill_lens(BatchLens* bl, const evlnPagedParams* p, const int* lens, const i
 }
 
 template <typename T>
-evlnStatus_t launch_combine(evlnHandle_t h, const CombineArgs& a, int D, bool paged, const BatchLens* bl,
+evlnStatus_t launch_combine(evlnHandle_t h, const CombineArgs& args, int D, bool paged, const BatchLens* bl,
                             cudaStream_t st)
 {
+    CombineArgs a = args;
+    a.div_g = make_fast_div((uint32_t)a.G);
+    a.div_chunk = make_fast_div((uint32_t)(a.chunk_tiles > 0 ? a.chunk_tiles : 1));
     dim3 grid(ceil_div(a.rows, 4), a.Hkv);
     if (paged) {
         if (D == 128) launch_pdl(combine_kernel<T, 128, true, BatchLens>, dim3(grid), dim3(128), 0, st, a, *bl);
@@ -526,6 +529,17 @@ evlnStatus_t evlnStepQRotSize(evlnHandle_t h, const evlnStepParams* p, size_t* b
     return EVLN_OK;
 }
 
+// The fields of RopeArgs that follow from the others (vec: elements per 16-byte vector).
+static void finish_rope_args(RopeArgs* a, int vec)
+{
+    a->G = a->Hq / a->Hkv;
+    a->div_g = make_fast_div((uint32_t)a->G);
+    a->vph_shift = 0;
+    while ((1 << a->vph_shift) < a->D / 2 / vec) ++a->vph_shift;
+    a->page_shift = 0;
+    while ((1 << a->page_shift) < a->page_size) ++a->page_shift;
+}
+
 static evlnStatus_t rope_append_impl(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
                                      const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok,
                                      void* q_rot, void* k_cache, void* v_cache, void* stream, const PackedMap& map)
@@ -555,6 +569,7 @@ static evlnStatus_t rope_append_impl(evlnHandle_t h, const evlnStepParams* p, co
     a.table = (const double2*)p->rope_table;
     a.table_first = p->rope_table_first_pos;
     a.map = map;
+    finish_rope_args(&a, p->dtype == EVLN_BF16 ? 8 : 4);
     NoLens nl = {};
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16)
@@ -737,6 +752,7 @@ evlnStatus_t evlnPagedRopeAppend(evlnHandle_t h, const evlnPagedParams* p, const
     a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
     a.num_new = total; a.batch = p->batch; a.page_size = p->page_size; a.max_pages = p->max_pages_per_seq;
     a.log2_theta = log2(p->rope_theta);
+    finish_rope_args(&a, 8);
     BatchLens bl;
     fill_lens(&bl, p, h_cache_lens, h_new_offsets);
     launch_pdl(rope_append_kernel<__nv_bfloat16, true, BatchLens>, dim3(total), dim3(256), 0, (cudaStream_t)stream, a, bl);
@@ -980,6 +996,7 @@ extern "C" evlnStatus_t evlnPackedForward(evlnHandle_t h, const evlnPackedParams
         a.log2_theta = log2(p->rope_theta);
         a.tail = 1;
         a.map = map_a;
+        finish_rope_args(&a, 8);
         launch_pdl(rope_append_kernel<__nv_bfloat16, true, BatchLens>, dim3(pl.n_act), dim3(256), 0, st, a, bl);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(h, e);

@@ -36,6 +36,12 @@ struct RopeArgs {
     int tail;               // batch mode without pages: K/V of new token m go to row m of k_cache / v_cache
                             // = buffers [Hkv, total new tokens, D] (the items' own tokens, not a shared cache)
     PackedMap map;          // where new token m sits in q_new / k_new / v_new (identity unless packed)
+    // derived by the host (finish_rope_args): the threads decode their work with shifts and one
+    // multiplication instead of integer divisions
+    int G;                  // Hq / Hkv
+    FastDiv div_g;
+    int vph_shift;          // log2 of the 16-byte vectors per half head vector (D/2 / V)
+    int page_shift;         // log2(page_size)
 };
 
 // cos/sin of pos * theta^(-2j/D): the one definition the append, gather and table kernels share
@@ -76,7 +82,7 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
 
     const int tok = blockIdx.x;           // index into the packed new tokens
     const int D = a.D, half = D / 2;
-    const int G = a.Hq / a.Hkv;
+    const int G = a.G;
 
     int b = 0, i = tok, L = a.cache_len, n_b = a.num_new;
     if (PAGED) {
@@ -103,8 +109,8 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
     long page_base = 0;     // paged: (page_id * Hkv) * page_size * D, slot within page
     int slot = 0;
     if (PAGED && !a.tail) {
-        int pg = a.page_table[(long)b * a.max_pages + (int)(pos / a.page_size)];
-        slot = (int)(pos % a.page_size);
+        int pg = a.page_table[(long)b * a.max_pages + (int)(pos >> a.page_shift)];
+        slot = (int)(pos & (a.page_size - 1));
         page_base = (long)pg * a.Hkv * a.page_size * D;
     }
     auto kv_row = [&](int g) -> long {
@@ -118,10 +124,10 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
     const T* k_tok = (const T*)a.k_new + src_tok * a.k_stride;
     const T* v_tok = (const T*)a.v_new + src_tok * a.v_stride;
 
-    const int vec_per_half = half / V;
-    const int q_items = a.Hq * vec_per_half;
-    const int k_items = a.Hkv * vec_per_half;
-    const int v_items = a.Hkv * (D / V);
+    const int vph = a.vph_shift, vpr = a.vph_shift + 1;       // vectors per half head vector / per head vector (log2)
+    const int q_items = a.Hq << vph;
+    const int k_items = a.Hkv << vph;
+    const int v_items = a.Hkv << vpr;
     const int items = q_items + k_items + v_items;
     const long rows_per_head = PAGED ? (long)lens.new_off[a.batch] * G : (long)a.num_new * G;
 
@@ -131,15 +137,15 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
         if (it < q_items + k_items) {
             const bool is_q = it < q_items;
             const int e = is_q ? it : it - q_items;
-            const int h = e / vec_per_half;
-            const int j0 = (e % vec_per_half) * V;
+            const int h = e >> vph;
+            const int j0 = (e & ((1 << vph) - 1)) * V;
             const T* src = (is_q ? q_tok : k_tok) + (long)h * D;
             r0 = *reinterpret_cast<const uint4*>(src + j0);
             r1 = *reinterpret_cast<const uint4*>(src + j0 + half);
         } else {
             const int e = it - q_items - k_items;
-            const int g = e / (D / V);
-            const int d0 = (e % (D / V)) * V;
+            const int g = e >> vpr;
+            const int d0 = (e & ((1 << vpr) - 1)) * V;
             r0 = *reinterpret_cast<const uint4*>(v_tok + (long)g * D + d0);
         }
     };
@@ -147,12 +153,12 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
         if (it < q_items + k_items) {
             const bool is_q = it < q_items;
             const int e = is_q ? it : it - q_items;
-            const int h = e / vec_per_half;
-            const int j0 = (e % vec_per_half) * V;
+            const int h = e >> vph;
+            const int j0 = (e & ((1 << vph) - 1)) * V;
             T* dst;
             if (is_q) {
-                const int g = h / G;
-                dst = (T*)a.q_rot + ((long)g * rows_per_head + (long)tok * G + (h % G)) * D;
+                const int g = (int)fast_div((uint32_t)h, a.div_g);
+                dst = (T*)a.q_rot + ((long)g * rows_per_head + (long)tok * G + (h - g * G)) * D;
             } else {
                 dst = (T*)a.k_cache + kv_row(h);
             }
@@ -174,8 +180,8 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
             *reinterpret_cast<uint4*>(dst + j0 + half) = out_hi_raw;
         } else {
             const int e = it - q_items - k_items;
-            const int g = e / (D / V);
-            const int d0 = (e % (D / V)) * V;
+            const int g = e >> vpr;
+            const int d0 = (e & ((1 << vpr) - 1)) * V;
             *reinterpret_cast<uint4*>((T*)a.v_cache + kv_row(g) + d0) = lo_raw;
         }
     };
