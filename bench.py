@@ -256,7 +256,12 @@ class PagedBatch:
         for b, t in enumerate(x["page_table"]):
             table[b, :len(t)] = torch.tensor(t, dtype=torch.int32)
         self.table = table.to(dev)
-        self.p = B.paged_params(Hq, Hkv, D, Bn, P, x["num_pages"], max_pages, cfg.rope_theta)
+        # one position table for 0 .. the longest episode: made once, like a model's RoPE cache
+        count = max(L + self.offs[b + 1] - self.offs[b] for b, L in enumerate(self.lens))
+        self.rope_table = torch.empty(B.evlnRopeTableBytes(D, count), dtype=torch.uint8, device=dev)
+        B.evlnRopeTable(handle, D, cfg.rope_theta, 0, count, self.rope_table)
+        self.p = B.paged_params(Hq, Hkv, D, Bn, P, x["num_pages"], max_pages, cfg.rope_theta,
+                                rope_table=self.rope_table, rope_table_first_pos=0, rope_table_count=count)
         total = self.offs[-1]
         wbytes = B.evlnPagedWorkspaceSize(handle, self.p, self.lens, self.offs)
         self.layers = []

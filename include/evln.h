@@ -105,6 +105,14 @@ typedef struct {
     int kv_chunk_tiles;      /* max 128-key tiles per work item; 0 = library heuristic       */
     float softmax_scale;     /* 0 -> 1/sqrt(D)                                               */
     double rope_theta;
+    /* Optional position table written by evlnRopeTable (NULL: the append kernel forms the angles
+     * itself).  It must cover the positions of every episode's new tokens, cache_len[b] ..
+     * cache_len[b] + n_b - 1: a serving host makes one table for positions 0 .. its longest
+     * context once, since the entries depend on head_dim and rope_theta only.  Results are
+     * bit-identical either way.                                                                */
+    const void* rope_table;
+    int rope_table_first_pos;
+    int rope_table_count;
 } evlnPagedParams;
 
 /* ---- handle, errors ------------------------------------------------------------------- */

@@ -51,7 +51,8 @@ class evlnPagedParams(Structure):
     _fields_ = [("struct_size", c_size_t), ("dtype", c_int), ("num_q_heads", c_int),
                 ("num_kv_heads", c_int), ("head_dim", c_int), ("batch", c_int),
                 ("page_size", c_int), ("num_pages", c_int), ("max_pages_per_seq", c_int),
-                ("kv_chunk_tiles", c_int), ("softmax_scale", c_float), ("rope_theta", c_double)]
+                ("kv_chunk_tiles", c_int), ("softmax_scale", c_float), ("rope_theta", c_double),
+                ("rope_table", c_void_p), ("rope_table_first_pos", c_int), ("rope_table_count", c_int)]
 
 
 class evlnPackedParams(Structure):
@@ -200,10 +201,12 @@ def step_params(dtype, num_q_heads, num_kv_heads, head_dim, cache_len, num_new, 
 
 
 def paged_params(num_q_heads, num_kv_heads, head_dim, batch, page_size, num_pages, max_pages_per_seq,
-                 rope_theta, softmax_scale=0.0, kv_chunk_tiles=0, dtype=EVLN_BF16) -> evlnPagedParams:
+                 rope_theta, softmax_scale=0.0, kv_chunk_tiles=0, dtype=EVLN_BF16, rope_table=None,
+                 rope_table_first_pos=0, rope_table_count=0) -> evlnPagedParams:
     return evlnPagedParams(ctypes.sizeof(evlnPagedParams), dtype, num_q_heads, num_kv_heads, head_dim,
                            batch, page_size, num_pages, max_pages_per_seq, kv_chunk_tiles, softmax_scale,
-                           rope_theta)
+                           rope_theta, _ptr(rope_table),
+                           int(rope_table_first_pos), int(rope_table_count))
 
 
 # ---- the entry points, by their C names ----------------------------------------------------

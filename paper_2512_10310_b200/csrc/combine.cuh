@@ -34,8 +34,6 @@ __global__ void __launch_bounds__(128)
 combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
 {
     constexpr int C = D / 32;
-    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t row = blockIdx.x * 4u + (uint32_t)warp;      // packed row within kv head (< 2^24, checked on the host)
     const int g = blockIdx.y;
@@ -62,10 +60,15 @@ combine_kernel(const CombineArgs a, const __grid_constant__ LensT lens)
 
     const long stride_s = (long)a.Hkv * a.rows;           // rows between consecutive splits
     const long prow0 = (long)g * a.rows + row;
+    // (so far launch parameters only: a row's warp knows its place before the partials exist)
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    constexpr int kPre = 4;
+    // (Letting every lane read all log-sum-exps of a row with few splits, so that the maximum and
+    // the weights need no shuffles, was measured slower: 3.85 against 3.45 us at the 7B step.)
     float my_lse = (lane < S) ? a.lse_part[prow0 + lane * stride_s] : -INFINITY;
     // the first partial rows do not depend on the weights: their loads go out with the lse load
-    constexpr int kPre = 4;
     float pre[kPre][C];
 #pragma unroll
     for (int s = 0; s < kPre; ++s) {

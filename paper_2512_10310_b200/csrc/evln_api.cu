@@ -250,6 +250,8 @@ evlnStatus_t check_paged_params(evlnHandle_t h, const evlnPagedParams* p, const 
         if (lens[b] < 0 || offs[b + 1] < offs[b]) return EVLN_INVALID_VALUE;
         const long tokens = (long)lens[b] + (offs[b + 1] - offs[b]);
         if ((tokens + p->page_size - 1) / p->page_size > p->max_pages_per_seq) return EVLN_CACHE_FULL;
+        if (!rope_table_covers(p->rope_table, p->rope_table_first_pos, p->rope_table_count, lens[b], offs[b + 1] - offs[b]))
+            return EVLN_INVALID_VALUE;
     }
     if ((long)offs[p->batch] * p->num_q_heads / p->num_kv_heads > (1 << 24)) return EVLN_NOT_SUPPORTED;
     return EVLN_OK;
@@ -347,6 +349,33 @@ evlnStatus_t launch_combine(evlnHandle_t h, const CombineArgs& args, int D, bool
     }
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
+}
+
+// The fields of RopeArgs that follow from the others (vec: elements per 16-byte vector).
+void finish_rope_args(RopeArgs* a, int vec)
+{
+    a->G = a->Hq / a->Hkv;
+    a->div_g = make_fast_div((uint32_t)a->G);
+    a->vph_shift = 0;
+    while ((1 << a->vph_shift) < a->D / 2 / vec) ++a->vph_shift;
+    a->page_shift = 0;
+    while ((1 << a->page_shift) < a->page_size) ++a->page_shift;
+}
+
+// The append kernel for `tokens` tokens.  Few enough to be one wave of two blocks per SM: one thread
+// per work item (in whole warps, at most kRopeThreadsMax).  Else 256 threads.
+template <typename T, bool PAGED, typename LensT>
+void launch_rope_append(evlnHandle_t h, const RopeArgs& a, int tokens, cudaStream_t st, const LensT& lens)
+{
+    const bool few = tokens <= 2 * h->num_sms;
+    int t = kRopeThreads;
+    if (few) {
+        const int items = ((a.Hq + a.Hkv) << a.vph_shift) + (a.Hkv << (a.vph_shift + 1));
+        t = (items + 31) / 32 * 32;
+        if (t > kRopeThreadsMax) t = kRopeThreadsMax;
+        if (t < 64) t = 64;
+    }
+    launch_pdl(rope_append_kernel<T, PAGED, LensT>, dim3(tokens), dim3(t), 0, st, a, lens);
 }
 
 evlnStatus_t noalloc_status_word(int** word);     // defined with the allocation-free variant below
@@ -529,17 +558,6 @@ evlnStatus_t evlnStepQRotSize(evlnHandle_t h, const evlnStepParams* p, size_t* b
     return EVLN_OK;
 }
 
-// The fields of RopeArgs that follow from the others (vec: elements per 16-byte vector).
-static void finish_rope_args(RopeArgs* a, int vec)
-{
-    a->G = a->Hq / a->Hkv;
-    a->div_g = make_fast_div((uint32_t)a->G);
-    a->vph_shift = 0;
-    while ((1 << a->vph_shift) < a->D / 2 / vec) ++a->vph_shift;
-    a->page_shift = 0;
-    while ((1 << a->page_shift) < a->page_size) ++a->page_shift;
-}
-
 static evlnStatus_t rope_append_impl(evlnHandle_t h, const evlnStepParams* p, const void* q_new, const void* k_new,
                                      const void* v_new, long q_stride_tok, long k_stride_tok, long v_stride_tok,
                                      void* q_rot, void* k_cache, void* v_cache, void* stream, const PackedMap& map)
@@ -573,9 +591,9 @@ static evlnStatus_t rope_append_impl(evlnHandle_t h, const evlnStepParams* p, co
     NoLens nl = {};
     cudaStream_t st = (cudaStream_t)stream;
     if (p->dtype == EVLN_BF16)
-        launch_pdl(rope_append_kernel<__nv_bfloat16, false, NoLens>, dim3(p->num_new), dim3(256), 0, st, a, nl);
+        launch_rope_append<__nv_bfloat16, false, NoLens>(h, a, p->num_new, st, nl);
     else
-        launch_pdl(rope_append_kernel<float, false, NoLens>, dim3(p->num_new), dim3(256), 0, st, a, nl);
+        launch_rope_append<float, false, NoLens>(h, a, p->num_new, st, nl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
@@ -752,10 +770,12 @@ evlnStatus_t evlnPagedRopeAppend(evlnHandle_t h, const evlnPagedParams* p, const
     a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads; a.D = p->head_dim;
     a.num_new = total; a.batch = p->batch; a.page_size = p->page_size; a.max_pages = p->max_pages_per_seq;
     a.log2_theta = log2(p->rope_theta);
+    a.table = (const double2*)p->rope_table;
+    a.table_first = p->rope_table_first_pos;
     finish_rope_args(&a, 8);
     BatchLens bl;
     fill_lens(&bl, p, h_cache_lens, h_new_offsets);
-    launch_pdl(rope_append_kernel<__nv_bfloat16, true, BatchLens>, dim3(total), dim3(256), 0, (cudaStream_t)stream, a, bl);
+    launch_rope_append<__nv_bfloat16, true, BatchLens>(h, a, total, (cudaStream_t)stream, bl);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? EVLN_OK : cuda_fail(h, e);
 }
@@ -997,7 +1017,7 @@ extern "C" evlnStatus_t evlnPackedForward(evlnHandle_t h, const evlnPackedParams
         a.tail = 1;
         a.map = map_a;
         finish_rope_args(&a, 8);
-        launch_pdl(rope_append_kernel<__nv_bfloat16, true, BatchLens>, dim3(pl.n_act), dim3(256), 0, st, a, bl);
+        launch_rope_append<__nv_bfloat16, true, BatchLens>(h, a, pl.n_act, st, bl);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return cuda_fail(h, e);
     }

@@ -6,10 +6,15 @@
 // into shared memory for all heads: from the caller's position table when there is one (the
 // table depends on the positions only, so a model makes it once per navigation step for all its
 // layers: rope_table_kernel below), else formed on the spot.  Phase 2: every thread moves 16-byte
-// vectors: rotated query halves to the kv-head-grouped q_rot scratch, rotated key halves and
-// the unchanged values to the token's cache slot; the loads of a thread's first vectors are
-// issued before the trigonometry is waited for.  HBM-bound: each element is read once and
-// written once with 128-bit accesses.
+// vectors (a work item is a pair of vectors (j.., j + D/2..) of a query or key head, or one vector
+// of a value head): rotated query halves to the kv-head-grouped q_rot scratch, rotated key halves
+// and the unchanged values to the token's cache slot; the loads of a thread's first item are issued
+// before the cos/sin are waited for.  HBM-bound by bytes (each element is read once and written
+// once with 128-bit accesses); at the sizes of a step it is one chain of latencies, which is why
+// nothing in it divides, and why a call of few tokens gets one thread per work item (all loads of
+// a token in flight at once).  (Letting every thread read the table entries of its own vector
+// instead of sharing them through shared memory was measured slower: 32 heads re-read the same 64
+// entries.)
 #pragma once
 
 #include "common.cuh"
@@ -70,13 +75,16 @@ rope_table_kernel(double2* table, int first_pos, int count, int D, double log2_t
 
 // LensT is BatchLens for the paged kernel and NoLens (a stub) for the contiguous one.
 
+// Block size: calls of few tokens (one wave of blocks) get one thread per work item, in whole warps,
+// at most kRopeThreadsMax; batches of thousands of tokens are bound by throughput and take 256.
+constexpr int kRopeThreadsMax = 384;
+constexpr int kRopeThreads = 256;
+
 template <typename T, bool PAGED, typename LensT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kRopeThreadsMax)
 rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
 {
     constexpr int V = VecTraits<T>::kVec;
-    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ double s_cos[128];
     __shared__ double s_sin[128];
 
@@ -97,10 +105,14 @@ rope_append_kernel(const RopeArgs a, const __grid_constant__ LensT lens)
         n_b = lens.new_off[b + 1] - lens.new_off[b];
     }
     const long pos = (long)L + i;
+    // (so far launch parameters only; what follows reads memory that earlier kernels may have written)
+    asm volatile("griddepcontrol.wait;" ::: "memory");          // programmatic dependent launch: inputs ready
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const double2* trow = a.table ? a.table + (pos - a.table_first) * half : nullptr;
 
     if (threadIdx.x < half) {
         const int j = threadIdx.x;
-        const double2 cs = a.table ? a.table[(pos - a.table_first) * half + j] : rope_cos_sin(pos, j, D, a.log2_theta);
+        const double2 cs = trow ? trow[j] : rope_cos_sin(pos, j, D, a.log2_theta);
         s_cos[j] = cs.x;
         s_sin[j] = cs.y;
     }

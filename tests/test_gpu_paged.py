@@ -22,7 +22,7 @@ def handle():
     B.evlnDestroy(h)
 
 
-def _gpu_paged(handle, cfg, x, kv_chunk_tiles=0):
+def _gpu_paged(handle, cfg, x, kv_chunk_tiles=0, with_table=False):
     dev = "cuda:0"
     Bn, P = len(x["cache_lens"]), cfg.page_size
     Hq, Hkv, D = cfg.num_q_heads, cfg.num_kv_heads, cfg.head_dim
@@ -41,8 +41,15 @@ def _gpu_paged(handle, cfg, x, kv_chunk_tiles=0):
             cnt = min(P, L - pi * P)
             k_pool[pg, :, :cnt] = x["k_pool"][pg, :cnt].to(dev).permute(1, 0, 2)
             v_pool[pg, :, :cnt] = x["v_pool"][pg, :cnt].to(dev).permute(1, 0, 2)
-    p = B.paged_params(Hq, Hkv, D, Bn, P, x["num_pages"], max_pages, cfg.rope_theta, kv_chunk_tiles=kv_chunk_tiles)
     lens, offs = x["cache_lens"], x["new_offsets"]
+    rope = {}
+    if with_table:
+        # one table for positions 0 .. the longest episode, as a serving host would keep
+        count = max(L + offs[b + 1] - offs[b] for b, L in enumerate(lens))
+        tbl = torch.empty(B.evlnRopeTableBytes(D, count), dtype=torch.uint8, device=dev)
+        B.evlnRopeTable(handle, D, cfg.rope_theta, 0, count, tbl)
+        rope = dict(rope_table=tbl, rope_table_first_pos=0, rope_table_count=count)
+    p = B.paged_params(Hq, Hkv, D, Bn, P, x["num_pages"], max_pages, cfg.rope_theta, kv_chunk_tiles=kv_chunk_tiles, **rope)
     total = offs[-1]
     q, k, v = (x[s].to(dev) for s in ("q_new", "k_new", "v_new"))
     q_rot = torch.empty(total * Hq * D * 2 + 256, dtype=torch.uint8, device=dev)
@@ -84,6 +91,25 @@ def test_paged_small_ragged_batch(handle):
                                          x["page_table"], lens, x["new_offsets"], cfg.rope_theta, storage="bf16")
         check_output("bf16", out, lse, ref_out, ref_lse)
         _check_pools(x, cfg, k_pool, v_pool, okp, ovp)
+
+
+def test_paged_position_table_gives_the_same_bits(handle):
+    # few tokens (threads read the table themselves) and many (through shared memory), against the
+    # kernel's own trigonometry: identical pools and outputs; a table that stops short is refused
+    for lens, news in (([0, 63, 64, 333, 1000], [70, 1, 129, 37, 196]), ([300, 2000, 1234, 77], [196, 196, 150, 64])):
+        cfg = dataclasses.replace(W.PAGED_B16, name="paged_table", batch=len(lens), seed=35)
+        x = W.make_paged_inputs(cfg, lens=lens, num_new=news)
+        a = _gpu_paged(handle, cfg, x)
+        b = _gpu_paged(handle, cfg, x, with_table=True)
+        for u, v in zip(a, b):
+            assert torch.equal(torch.nan_to_num(u.float(), nan=-7.0), torch.nan_to_num(v.float(), nan=-7.0))
+    D = cfg.head_dim
+    tbl = torch.empty(B.evlnRopeTableBytes(D, 100), dtype=torch.uint8, device="cuda:0")
+    p = B.paged_params(cfg.num_q_heads, cfg.num_kv_heads, D, 1, cfg.page_size, 8, 8, cfg.rope_theta,
+                       rope_table=tbl, rope_table_first_pos=0, rope_table_count=100)
+    with pytest.raises(B.EvlnError) as e:
+        B.evlnPagedWorkspaceSize(handle, p, [90], [0, 20])          # positions 90..109, table ends at 99
+    assert e.value.status == B.EVLN_INVALID_VALUE
 
 
 def test_paged_equals_contiguous_on_device(handle):

@@ -38,15 +38,17 @@ def test_struct_sizes_match_the_header_layout(tmp_path):
     src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "evln.h"\n'
                    'int main(void) { printf("%zu %zu %zu %zu %zu\\n", sizeof(evlnStepParams), sizeof(evlnPagedParams), '
                    'sizeof(evlnGatherParams), offsetof(evlnStepParams, rope_table), offsetof(evlnGatherParams, rope_table)); '
+                   'printf("%zu\\n", offsetof(evlnPagedParams, rope_table)); '
                    'return 0; }\n')
     exe = tmp_path / "sizes"
     subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
-    step, paged, gather, off_step, off_gather = map(int, subprocess.check_output([str(exe)]).split())
+    step, paged, gather, off_step, off_gather, off_paged = map(int, subprocess.check_output([str(exe)]).split())
     assert ctypes.sizeof(B.evlnStepParams) == step == 72
-    assert ctypes.sizeof(B.evlnPagedParams) == paged == 56
+    assert ctypes.sizeof(B.evlnPagedParams) == paged == 72
     assert ctypes.sizeof(B.evlnGatherParams) == gather == 56
     assert B.evlnStepParams.rope_table.offset == off_step
     assert B.evlnGatherParams.rope_table.offset == off_gather
+    assert B.evlnPagedParams.rope_table.offset == off_paged
 
 
 def test_page_table_check_on_the_host(lib):
