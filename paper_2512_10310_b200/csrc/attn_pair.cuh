@@ -242,6 +242,20 @@ __device__ __forceinline__ void exp32(const uint32_t* s, uint32_t (&packed)[16],
     }
 }
 
+// The largest of a row's first 32 scores of a score buffer (columns 0 .. lim visible), scaled: what the
+// publisher of the row's reference computes, for a thread that would rather read the scores itself
+// than wait for the publication.  Kept out of line so that it does not disturb the tile loop's code.
+__device__ __noinline__ float first_block_reference(uint32_t taddr, int lim, float scale_log2)
+{
+    uint32_t f[32];
+    ptx::tmem_ld32(taddr, f);
+    ptx::tmem_ld_wait();
+    if (!__all_sync(0xffffffffu, lim >= 63)) mask32(f, lim);
+    float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
+    rowmax32(f, x0, x1, x2, x3);
+    return fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)) * scale_log2;
+}
+
 // --- work decoding ------------------------------------------------------------------------
 
 struct WorkItem {
@@ -789,7 +803,19 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
         // row sees no key of this split, since the visible keys of a row are a prefix).  The
         // thread that owns those columns reads it off and publishes it; nobody can ask for a new
         // reference before, so the other threads of the row simply wait for it.
-        if (part != 0) {
+        if (part == 1 && ntiles > 0) {
+            // The other half of the first tile's group does not wait for the publisher: it reads the
+            // same 32 scores itself (the buffer is not given back before all of the group's warps
+            // have arrived) and gets the same maximum, ~1 K cycles before the published one could
+            // reach it: the first product starts that much earlier.
+            ok = warp_wait(bar_s_full, 0, kDevTimeoutSoftmaxS, a.status, s_abort, lane);
+            if (ok) {
+                ptx::fence_after_sync();
+                int lim0 = bound - w.j0 * kTileN;
+                if (TAIL) lim0 = w.j0 < nct ? w.L - 1 - w.j0 * kTileN : bound - (w.j0 - nct) * kTileN;
+                m_ref = first_block_reference(t_lane, lim0, a.scale_log2);
+            }
+        } else if (part != 0) {
             ok = warp_wait(bar_ref + 8 * quarter, 0, kDevTimeoutSoftmaxX, a.status, s_abort, lane);
             if (ok) m_ref = s_ref[r_tile];
         }
