@@ -26,7 +26,10 @@
  *    the cudaError_t value.
  *  - The library does not advance L: the caller passes the pre-step cache length to all
  *    three calls of a step and adds n afterwards.
- *  - For fixed parameters the split schedule is fixed, so results are bitwise reproducible.
+ *  - For fixed parameters the split schedule is fixed, so results are bitwise reproducible, with
+ *    one exception in the tensor-core kernel: when a score exceeds the maximum of its row's first
+ *    KV tile by more than a factor 2^64, the row's softmax reference moves, and where it moves to
+ *    depends on which of the row's threads noticed first; results then agree to rounding only.
  *  - One handle per host thread.  There is no CPU fallback.
  *
  * Layouts (D = head_dim, G = num_q_heads / num_kv_heads, query head h uses kv head h / G)

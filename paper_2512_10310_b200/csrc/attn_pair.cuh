@@ -471,38 +471,21 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
 
     auto on_cta0 = [&](uint32_t bar) -> uint32_t { return CTAS == 2 ? ptx::map_to_cta(bar, 0) : bar; };
 
-    // Registers go where the work is: the warpgroup of the producer and the issuers gives most of its
-    // share back, the two softmax warpgroups (128 scores per thread in flight) take it.
-    if (warp < 4) {
-    ptx::setmaxnreg_dec<kRegsIssue>();
-    if (warp == 0) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            // everything this CTA reads or writes in global memory follows this thread's loads, so
-            // one wait here orders the whole CTA after the kernels it depends on
-            ptx::grid_dependency_wait();
+    // ---- the TMA producer's tools (used by one thread of warp 0) ----
+    bool ok_prod = true;
             auto expect = [&](uint32_t bar, uint32_t bytes) {
                 if (CTAS == 2) ptx::mbar_expect_tx_cluster(bar, bytes); else ptx::mbar_expect_tx(bar, bytes);
             };
             auto tma3 = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
                 if (CTAS == 2) ptx::tma_load_3d_pair(dst, map, bar, x, y, z); else ptx::tma_load_3d(dst, map, bar, x, y, z);
             };
-            {
-                const uint32_t q_full0 = on_cta0(bar_q_full);
-                const uint32_t dst = smem_base + kSmemQOff;
-                const int qrow = w.row_base + row0;
-                expect(q_full0, kTileBytes);
-                tma3(dst, &tm_q, q_full0, 0, qrow, w.g);
-                tma3(dst + kHalfBytes, &tm_q, q_full0, 64, qrow, w.g);
-            }
-            bool ok = true;
             // K tile j.  Pair: this CTA's half, keys [128 j + 64 rank, +64), all channels (two 64-channel
             // blocks of 64 keys).  Alone: the whole tile (two 64-channel blocks of 128 keys).
             auto load_k = [&](int jj) {
                 const int stage = jj % kKStages;
                 if (jj >= kKStages)
-                    ok = wait_bounded(bar_k_empty + 8 * stage, ((jj / kKStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
-                if (!ok) return;
+                    ok_prod = wait_bounded(bar_k_empty + 8 * stage, ((jj / kKStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
+                if (!ok_prod) return;
                 const uint32_t dst = smem_base + kSmemKOff + stage * kStageBytes;
                 const uint32_t bar = on_cta0(bar_k_full + 8 * stage);
                 const int j = w.j0 + jj;
@@ -534,8 +517,8 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
             auto load_v = [&](int jj) {
                 const int stage = jj % kVStages;
                 if (jj >= kVStages)
-                    ok = wait_bounded(bar_v_empty + 8 * stage, ((jj / kVStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
-                if (!ok) return;
+                    ok_prod = wait_bounded(bar_v_empty + 8 * stage, ((jj / kVStages) & 1) ^ 1, kDevTimeoutProducer, a.status, s_abort);
+                if (!ok_prod) return;
                 const uint32_t dst = smem_base + kSmemVOff + stage * kStageBytes;
                 const uint32_t bar = on_cta0(bar_v_full + 8 * stage);
                 const int j = w.j0 + jj;
@@ -556,14 +539,40 @@ __device__ __forceinline__ void attn_tc_body(const CUtensorMap& tm_q, const CUte
                     ptx::tma_load_4d_pair(dst + 8192, &tm_v, bar, 64 * (int)rank, 0, w.g, pt[p1]);
                 }
             };
-            // in the order the MMAs consume them: K_0, K_1, then V_j, K_{j+2}
-            const int pre = ntiles < kScoreBufs ? ntiles : kScoreBufs;
-            for (int jj = 0; jj < pre && ok; ++jj) load_k(jj);
-            for (int jj = 0; jj < ntiles && ok; ++jj) {
-                load_v(jj);
-                if (ok && jj + kScoreBufs < ntiles) load_k(jj + kScoreBufs);
+
+    // The producer's first loads (Q, then the K tiles of the first scores) go out before the warps
+    // change their register shares: that hand-over is a rendezvous of the whole warpgroup, and the
+    // loads' latency is the longest item on the way to the first MMA.
+    const int pre_k = ntiles < kScoreBufs ? ntiles : kScoreBufs;
+    if (warp == 0 && lane == 0) {
+        // everything this CTA reads or writes in global memory follows this thread's loads, so
+        // one wait here orders the whole CTA after the kernels it depends on
+        ptx::grid_dependency_wait();
+            {
+                const uint32_t q_full0 = on_cta0(bar_q_full);
+                const uint32_t dst = smem_base + kSmemQOff;
+                const int qrow = w.row_base + row0;
+                expect(q_full0, kTileBytes);
+                tma3(dst, &tm_q, q_full0, 0, qrow, w.g);
+                tma3(dst + kHalfBytes, &tm_q, q_full0, 64, qrow, w.g);
             }
-            if (!ok || *s_abort) {
+        for (int jj = 0; jj < pre_k; ++jj) load_k(jj);
+    }
+    __syncwarp();            // (the register hand-over below wants whole warps)
+
+    // Registers go where the work is: the warpgroup of the producer and the issuers gives most of its
+    // share back, the two softmax warpgroups (128 scores per thread in flight) take it.
+    if (warp < 4) {
+    ptx::setmaxnreg_dec<kRegsIssue>();
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            // in the order the MMAs consume them: (K_0, K_1 are on their way,) then V_j, K_{j+2}
+            for (int jj = 0; jj < ntiles && ok_prod; ++jj) {
+                load_v(jj);
+                if (ok_prod && jj + kScoreBufs < ntiles) load_k(jj + kScoreBufs);
+            }
+            if (!ok_prod || *s_abort) {
                 // give this CTA's loads in flight time to land before the pair may leave
                 const long long t0 = clock64();
                 while (clock64() - t0 < 400000) { }
